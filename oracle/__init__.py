@@ -1,0 +1,236 @@
+"""CPU oracle for the lognormal gradient-compression path -- TEST INFRASTRUCTURE.
+
+Thin ctypes access to ``lgn_oracle.c`` (plain scalar C, fp64).  Only the tests,
+the smoke check and the benchmark's CPU-baseline leg import this package.  It
+imports nothing from the CUDA package and shares no code with it.
+
+Arrays are numpy: float32 for fp32 tensors, uint16 (raw bfloat16 bit patterns)
+for bf16 tensors.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "lgn_oracle.c")
+_LIB = os.path.join(_HERE, "liblgn_oracle.so")
+
+F32, BF16 = 0, 1
+ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with the host C compiler (no fast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-fno-fast-math",
+             _SRC, "-o", _LIB, "-lm"])
+    return _LIB
+
+
+class _Stats(C.Structure):
+    _fields_ = [("n", C.c_uint64), ("nnz", C.c_uint64), ("mu", C.c_double),
+                ("sigma", C.c_double), ("zero_frac", C.c_double)]
+
+
+_lib = None
+
+
+def _L():
+    global _lib
+    if _lib is None:
+        lib = C.CDLL(build())
+        u32, u64, i32, dbl, vp = C.c_uint32, C.c_uint64, C.c_int, C.c_double, C.c_void_p
+        lib.orc_stats.argtypes = [vp, u64, i32, C.POINTER(_Stats)]
+        lib.orc_stats.restype = None
+        lib.orc_philox4x32_10.argtypes = [vp, vp, vp]
+        lib.orc_philox4x32_10.restype = None
+        lib.orc_rand32.argtypes = [u64, u64]
+        lib.orc_rand32.restype = u32
+        lib.orc_rand32_fill.argtypes = [u64, u64, u64, vp]
+        lib.orc_rand32_fill.restype = None
+        lib.orc_sparsity_of.argtypes = [dbl, dbl]
+        lib.orc_sparsity_of.restype = dbl
+        lib.orc_threshold.argtypes = [dbl, dbl, dbl, dbl, C.POINTER(dbl)]
+        lib.orc_threshold.restype = i32
+        lib.orc_snap_tau.argtypes = [dbl, i32]
+        lib.orc_snap_tau.restype = dbl
+        lib.orc_prune_one.argtypes = [dbl, dbl, u32]
+        lib.orc_prune_one.restype = dbl
+        lib.orc_prune_with_bits.argtypes = [vp, vp, u64, i32, dbl, vp]
+        lib.orc_prune_with_bits.restype = None
+        lib.orc_prune.argtypes = [vp, vp, u64, i32, dbl, u64, u64]
+        lib.orc_prune.restype = None
+        lib.orc_expected_rel_err.argtypes = [dbl, i32, i32]
+        lib.orc_expected_rel_err.restype = dbl
+        lib.orc_fp_format.argtypes = [dbl, dbl, u64, i32, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+        lib.orc_fp_format.restype = i32
+        lib.orc_quantize_one.argtypes = [dbl, i32, i32, i32, i32, u32]
+        lib.orc_quantize_one.restype = u32
+        lib.orc_decode.argtypes = [u32, i32, i32, i32]
+        lib.orc_decode.restype = dbl
+        lib.orc_quantize_with_bits.argtypes = [vp, vp, u64, i32, i32, i32, i32, i32, vp]
+        lib.orc_quantize_with_bits.restype = None
+        lib.orc_quantize.argtypes = [vp, vp, u64, i32, i32, i32, i32, i32, u64, u64]
+        lib.orc_quantize.restype = None
+        lib.orc_packed_bytes.argtypes = [u64, i32]
+        lib.orc_packed_bytes.restype = u64
+        lib.orc_pack.argtypes = [vp, u64, i32, vp]
+        lib.orc_pack.restype = None
+        lib.orc_unpack.argtypes = [vp, u64, i32, vp]
+        lib.orc_unpack.restype = None
+        lib.orc_count_zeros.argtypes = [vp, u64, i32]
+        lib.orc_count_zeros.restype = u64
+        _lib = lib
+    return _lib
+
+
+def _dtype_of(g: np.ndarray) -> int:
+    if g.dtype == np.float32:
+        return F32
+    if g.dtype == np.uint16:
+        return BF16
+    raise TypeError("oracle tensors are float32 or uint16 (bfloat16 bits), got %s" % g.dtype)
+
+
+def _flat(g: np.ndarray) -> np.ndarray:
+    return np.ascontiguousarray(g).reshape(-1)
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+# --------------------------------------------------------------------------- stats
+def stats(g: np.ndarray) -> dict:
+    """nnz, mu, sigma of ln|g| over the nonzero entries; zero fraction l."""
+    g = _flat(g)
+    st = _Stats()
+    _L().orc_stats(_ptr(g), g.size, _dtype_of(g), C.byref(st))
+    return {"n": st.n, "nnz": st.nnz, "mu": st.mu, "sigma": st.sigma, "zero_frac": st.zero_frac}
+
+
+# --------------------------------------------------------------------------- rng
+def philox4x32_10(ctr, key):
+    c = np.asarray(ctr, dtype=np.uint32)
+    k = np.asarray(key, dtype=np.uint32)
+    o = np.zeros(4, dtype=np.uint32)
+    _L().orc_philox4x32_10(_ptr(c), _ptr(k), _ptr(o))
+    return o
+
+
+def rand32(seed: int, i: int) -> int:
+    return int(_L().orc_rand32(seed, i))
+
+
+def rand32_fill(seed: int, first: int, n: int) -> np.ndarray:
+    o = np.zeros(n, dtype=np.uint32)
+    _L().orc_rand32_fill(seed, first, n, _ptr(o))
+    return o
+
+
+# --------------------------------------------------------------------------- threshold / prune
+def sparsity_of(u: float, sigma: float) -> float:
+    """Eq. 8: expected pruned fraction at threshold alpha = e^(mu+u)."""
+    return float(_L().orc_sparsity_of(u, sigma))
+
+
+def threshold(mu: float, sigma: float, zero_frac: float, S: float) -> float:
+    tau = C.c_double()
+    rc = _L().orc_threshold(mu, sigma, zero_frac, S, C.byref(tau))
+    if rc != 0:
+        raise ValueError("orc_threshold: invalid argument")
+    return tau.value
+
+
+def snap_tau(tau: float, dtype: int) -> float:
+    return float(_L().orc_snap_tau(tau, dtype))
+
+
+def prune_one(x: float, tau_used: float, h: int) -> float:
+    return float(_L().orc_prune_one(x, tau_used, h))
+
+
+def prune_with_bits(g: np.ndarray, tau_used: float, h: np.ndarray) -> np.ndarray:
+    g = _flat(g)
+    h = np.ascontiguousarray(h, dtype=np.uint32)
+    assert h.size == g.size
+    out = np.empty_like(g)
+    _L().orc_prune_with_bits(_ptr(g), _ptr(out), g.size, _dtype_of(g), tau_used, _ptr(h))
+    return out
+
+
+def prune(g: np.ndarray, tau_used: float, seed: int, first: int = 0) -> np.ndarray:
+    g = _flat(g)
+    out = np.empty_like(g)
+    _L().orc_prune(_ptr(g), _ptr(out), g.size, _dtype_of(g), tau_used, seed, first)
+    return out
+
+
+# --------------------------------------------------------------------------- format / quantize
+def expected_rel_err(sigma: float, n1: int, n2: int) -> float:
+    """Eq. 4 for n1 mantissa bits and n2 exponent bits."""
+    return float(_L().orc_expected_rel_err(sigma, n1, n2))
+
+
+def fp_format(mu: float, sigma: float, nnz: int, nbits: int) -> dict:
+    e, m, s = C.c_int(), C.c_int(), C.c_int()
+    rc = _L().orc_fp_format(mu, sigma, nnz, nbits, C.byref(e), C.byref(m), C.byref(s))
+    if rc != 0:
+        raise ValueError("orc_fp_format: nbits outside 4..8")
+    return {"nbits": nbits, "exp_bits": e.value, "man_bits": m.value, "scale_exp": s.value}
+
+
+def quantize_one(x: float, n2: int, n1: int, e_s: int, rounding: int, h: int = 0) -> int:
+    return int(_L().orc_quantize_one(x, n2, n1, e_s, rounding, h))
+
+
+def decode(code: int, n2: int, n1: int, e_s: int) -> float:
+    return float(_L().orc_decode(code, n2, n1, e_s))
+
+
+def quantize_with_bits(g, n2, n1, e_s, rounding, h=None) -> np.ndarray:
+    g = _flat(g)
+    codes = np.empty(g.size, dtype=np.uint8)
+    hp = None
+    if h is not None:
+        h = np.ascontiguousarray(h, dtype=np.uint32)
+        assert h.size == g.size
+        hp = _ptr(h)
+    _L().orc_quantize_with_bits(_ptr(g), _ptr(codes), g.size, _dtype_of(g), n2, n1, e_s, rounding, hp)
+    return codes
+
+
+def quantize(g, n2, n1, e_s, rounding, seed=0, first=0) -> np.ndarray:
+    """One code per byte (unpacked)."""
+    g = _flat(g)
+    codes = np.empty(g.size, dtype=np.uint8)
+    _L().orc_quantize(_ptr(g), _ptr(codes), g.size, _dtype_of(g), n2, n1, e_s, rounding, seed, first)
+    return codes
+
+
+def packed_bytes(n: int, nbits: int) -> int:
+    return int(_L().orc_packed_bytes(n, nbits))
+
+
+def pack(codes: np.ndarray, nbits: int) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    out = np.zeros(packed_bytes(codes.size, nbits), dtype=np.uint8)
+    _L().orc_pack(_ptr(codes), codes.size, nbits, _ptr(out))
+    return out
+
+
+def unpack(packed: np.ndarray, n: int, nbits: int) -> np.ndarray:
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    codes = np.empty(n, dtype=np.uint8)
+    _L().orc_unpack(_ptr(packed), n, nbits, _ptr(codes))
+    return codes
+
+
+def count_zeros(g: np.ndarray) -> int:
+    g = _flat(g)
+    return int(_L().orc_count_zeros(_ptr(g), g.size, _dtype_of(g)))
