@@ -1,0 +1,198 @@
+/*
+ * lgn.h -- C ABI of the lognormal neural-gradient compression library for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library runs, per gradient tensor, the path of "Neural gradients are
+ * near-lognormal: improved quantized and sparse training" (arXiv 2006.08173):
+ *
+ *   statistics of ln|g| over the nonzero entries  (Section 3; Appendix A.8, A.9 step 3)
+ *     -> closed form: pruning threshold for a requested sparsity (Eq. 6-8; A.9 steps 1-2)
+ *                  or n-bit floating-point split and scale       (Eq. 4; Algorithm 1)
+ *     -> elementwise pass: stochastic pruning (Eq. 5) or FP quantisation (Eq. 1-2)
+ *
+ * Conventions that hold for every entry point
+ *  - "device" pointers are CUDA device addresses on the current device, owned
+ *    by the caller for the whole call and until the work enqueued on `stream`
+ *    has finished.  "host" pointers are ordinary process memory, read or
+ *    written before the call returns.
+ *  - The library allocates no device memory and keeps no state between calls,
+ *    except the entry points that say otherwise.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *    All device work is enqueued on it and the call returns without waiting.
+ *  - Tensors are contiguous and are treated as flat arrays of n elements; the
+ *    element index used for randomness is the flat index.
+ *  - Tensor base addresses (g, out, codes, workspace, result arrays) must be
+ *    16-byte aligned.  Input and output buffers must not overlap.
+ *  - Inputs must be finite.  +0 and -0 both count as zero.
+ *  - Argument errors are found on the host and returned before anything is
+ *    enqueued.  A CUDA error at enqueue time is returned as LGN_ERR_CUDA.
+ *  - Same inputs, seed and arguments give bitwise the same outputs and the same
+ *    statistics on every run.
+ */
+#ifndef LGN_H
+#define LGN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LGN_OK              = 0,
+    LGN_ERR_INVALID_ARG = 1,  /* null/misaligned pointer, S outside [0,1), bad enum, ... */
+    LGN_ERR_UNSUPPORTED = 2,  /* nbits outside 4..8, tensor too large                     */
+    LGN_ERR_WORKSPACE   = 3,  /* workspace smaller than lgn_workspace_bytes() says        */
+    LGN_ERR_CUDA        = 4,  /* the CUDA runtime refused a launch or copy                */
+    LGN_ERR_TIMEOUT     = 5   /* a bounded device-side wait ran out (per-layer status)    */
+} lgn_status;
+
+typedef enum { LGN_F32 = 0, LGN_BF16 = 1 } lgn_dtype;
+typedef enum { LGN_ROUND_NEAREST = 0, LGN_ROUND_STOCHASTIC = 1 } lgn_rounding;
+typedef enum { LGN_MODE_PRUNE = 0, LGN_MODE_QUANTIZE = 1 } lgn_mode;
+
+/* Lognormal statistics of one tensor (Section 3: magnitudes, zeros left out). */
+typedef struct {
+    uint64_t n;        /* elements                                               */
+    uint64_t nnz;      /* elements != 0                                          */
+    double   sum_ln;   /* sum of ln|g| over the nonzero elements                 */
+    double   sum_ln2;  /* sum of (ln|g|)^2 over the same                         */
+    double   mu;       /* sum_ln / nnz                      (0 when nnz == 0)    */
+    double   sigma;    /* population standard deviation of ln|g| (0 when nnz==0) */
+} lgn_stats_t;
+
+/* An n-bit floating-point format: 1 sign bit, exp_bits, man_bits, and the
+ * per-layer power-of-two scale of Algorithm 1 (values are divided by
+ * 2^scale_exp before quantisation).  1 + exp_bits + man_bits == nbits. */
+typedef struct {
+    int32_t nbits;      /* 4..8                    */
+    int32_t exp_bits;   /* n2, 1..nbits-1          */
+    int32_t man_bits;   /* n1, 0..nbits-2          */
+    int32_t scale_exp;  /* e_s                     */
+} lgn_fp_format_t;
+
+/* Text for a status code (static storage). */
+const char *lgn_status_string(lgn_status s);
+
+/* Device workspace, in bytes, that lgn_stats (num_layers = 1) or
+ * lgn_compress_layers needs for tensors of these element counts.
+ * n_per_layer: host.  Returns 0 if num_layers < 0 or a tensor is too large. */
+size_t lgn_workspace_bytes(const uint64_t *n_per_layer, int num_layers);
+
+/* Bytes of the packed code stream of n codes of nbits each:
+ * ceil(n*nbits/8) rounded up to a multiple of 4.  0 for nbits outside 4..8. */
+size_t lgn_codes_bytes(uint64_t n, int nbits);
+
+/* Statistics pass (Section 3; Appendix A.8 "mean and standard deviation of
+ * the input", A.9 step 3): nnz, and the mean and population standard deviation
+ * of the natural log of |g| over the nonzero elements.
+ *   g        device, n elements of dt, read only
+ *   out_dev  device, one lgn_stats_t, written when the stream reaches the call
+ *   ws       device scratch of at least lgn_workspace_bytes(&n, 1) bytes;
+ *            contents before and after are meaningless
+ * The logarithm is evaluated in fp32 (base-2 hardware approximation), summed
+ * in short fp32 runs and then in fp64, and combined across the grid in a fixed
+ * order: deterministic, within 1e-5 relative of an fp64 evaluation.
+ * n == 0 writes all zeros. */
+lgn_status lgn_stats(const void *g, uint64_t n, lgn_dtype dt, lgn_stats_t *out_dev,
+                     void *ws, size_t ws_bytes, void *stream);
+
+/* Sparsity -> threshold (Eq. 8 solved for alpha; Appendix A.9 steps 1-2).
+ * Host only, no CUDA call.
+ *   mu, sigma  lognormal parameters of the nonzero part
+ *   zero_frac  l, fraction of the tensor that is exactly zero, in [0,1]
+ *   S          requested fraction of zeros in the OUTPUT tensor, in [0,1)
+ *   tau        host, receives alpha (fp64, not yet rounded to the tensor type)
+ * The nonzero part has to reach S' = (S - l)/(1 - l); S' <= 0 or l == 1 gives
+ * tau = 0 (no pruning).  sigma is clamped to [1e-6, 25]. */
+lgn_status lgn_threshold(double mu, double sigma, double zero_frac, double S, double *tau);
+
+/* The threshold as the pruning kernel holds it: tau rounded to the tensor's
+ * storage type (ties to even; bf16 via fp32) and clamped to the largest finite
+ * value.  Host only.  Returns NaN for a negative or NaN tau or a bad dtype. */
+double lgn_snap_threshold(double tau, lgn_dtype dt);
+
+/* Optimal exponent/mantissa split and scale (Eq. 4 minimised over the integer
+ * splits n1 + n2 = nbits - 1, n2 >= 1; ties to the smaller n2) and the layer
+ * scale e_s = floor(mu/ln 2 + 1/2).  Host only.  Eq. 4 is read with the
+ * standard deviation of log2|g|, sigma/ln 2, and mantissa step 2^-n1.
+ *   fmt  host, receives the format.  sigma is clamped to [1e-6, 25]. */
+lgn_status lgn_fp_format(double mu, double sigma, int nbits, lgn_fp_format_t *fmt);
+
+/* Stochastic pruning with a given threshold (Eq. 5): the steady-state call
+ * between refreshes of the statistics.
+ *   g, out  device, n elements of dt; out has the same type and layout
+ *   tau     alpha >= 0; the kernel uses lgn_snap_threshold(tau, dt)
+ *   seed    element i draws eps_i = (r_i >> 9) / 2^23 where r_i is word i mod 4 of
+ *           Philox4x32-10 with key = (seed low, seed high), counter = (i/4 low,
+ *           i/4 high, 0, 0)
+ * |g_i| > alpha -> g_i;  fl32(alpha*eps_i) <= |g_i| <= alpha -> sign(g_i)*alpha;
+ * otherwise +0.  Zeros stay +0. */
+lgn_status lgn_prune(const void *g, void *out, uint64_t n, lgn_dtype dt, double tau,
+                     uint64_t seed, void *stream);
+
+/* FP quantisation with a given format (Eq. 1-2, Algorithm 1) into packed codes.
+ *   g      device, n elements of dt
+ *   codes  device, lgn_codes_bytes(n, fmt->nbits) bytes, all of them written:
+ *          a little-endian bit stream, code i in bits [i*nbits, (i+1)*nbits),
+ *          code = [sign | exponent field | mantissa], unused tail bits zero
+ *   fmt    host
+ *   seed   as in lgn_prune; used only with LGN_ROUND_STOCHASTIC
+ * With x' = x / 2^scale_exp = M * 2^E, E_max = 2^(exp_bits-1):
+ *   E >= E_max  (before rounding) -> largest code;
+ *   E <= -E_max (before rounding) -> 0 (nearest) or, stochastic, the smallest
+ *                normal with probability floor(2^24 |x'| / 2^(1-E_max)) / 2^24;
+ *   else M rounded to man_bits (nearest: ties to the even mantissa; stochastic:
+ *   top 23-man_bits bits of r_i added below the kept bits, then truncated),
+ *   a carry out of M moves to E, and E reaching E_max gives the largest code.
+ * Exponent field = E + E_max (1..2^exp_bits-1); field 0 encodes zero.
+ * A code decodes to (-1)^s (1 + m/2^man_bits) 2^(field - E_max + scale_exp). */
+lgn_status lgn_quantize(const void *g, void *codes, uint64_t n, lgn_dtype dt,
+                        const lgn_fp_format_t *fmt, lgn_rounding rounding,
+                        uint64_t seed, void *stream);
+
+/* One tensor of a grouped call. */
+typedef struct {
+    const void  *g;          /* device, n elements of dt                                  */
+    void        *out;        /* device: n elements of dt (prune) or lgn_codes_bytes(n,nbits) */
+    uint64_t     n;
+    int32_t      dt;         /* lgn_dtype                                                  */
+    int32_t      mode;       /* lgn_mode                                                   */
+    double       S;          /* prune: requested output sparsity in [0,1)                  */
+    int32_t      nbits;      /* quantize: 4..8                                             */
+    int32_t      rounding;   /* quantize: lgn_rounding                                     */
+    uint64_t     seed;
+    int32_t      use_override;   /* nonzero: use mu_override/sigma_override in the closed  */
+    int32_t      reserved;       /* form instead of the measured mu/sigma (nnz and the     */
+    double       mu_override;    /* zero fraction are always the measured ones)            */
+    double       sigma_override;
+} lgn_layer_t;
+
+typedef struct {
+    lgn_stats_t      stats;   /* measured, whatever the override says                     */
+    double           tau;     /* prune: the threshold used (already snapped); else 0       */
+    lgn_fp_format_t  fmt;     /* quantize: the format used; else zeros                     */
+    int32_t          status;  /* lgn_status of this layer (LGN_ERR_TIMEOUT: output invalid) */
+    int32_t          reserved;
+} lgn_layer_result_t;
+
+/* The whole path for a list of tensors in one kernel launch (plus one tiny
+ * set-up launch): statistics -> closed form on the device -> apply, per layer,
+ * with per-layer sparsity or bit-width (Section 5.3: different sparsity levels
+ * at different layers).  Tiles of all layers go through one work queue; a
+ * layer's apply tiles start as soon as its own statistics are complete, so a
+ * tensor that fits in L2 is still there when it is read the second time.
+ *   layers       host array of num_layers descriptors (copied before return)
+ *   results_dev  device array of num_layers results
+ *   ws           device scratch, lgn_workspace_bytes(n_per_layer, num_layers)
+ * Device-side waits are bounded; if one runs out the layer's status is
+ * LGN_ERR_TIMEOUT and the kernel still ends. */
+lgn_status lgn_compress_layers(const lgn_layer_t *layers, int num_layers,
+                               lgn_layer_result_t *results_dev,
+                               void *ws, size_t ws_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LGN_H */

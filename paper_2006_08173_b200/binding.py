@@ -1,0 +1,230 @@
+"""ctypes binding of ``liblgn.so`` (declared in ``include/lgn.h``).
+
+Argument marshalling only: torch supplies device memory and the current CUDA
+stream, every step of the path runs in the library's kernels.  There is no CPU
+fallback: if the shared library is missing or cannot be loaded, importing this
+module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "liblgn.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} not found: build it with `python -m paper_2006_08173_b200.build` "
+        "(nvcc, sm_100a); this package has no CPU fallback")
+_lib = C.CDLL(LIB_PATH)
+
+LGN_OK = 0
+F32, BF16 = 0, 1
+ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
+MODE_PRUNE, MODE_QUANTIZE = 0, 1
+
+
+class StatsT(C.Structure):
+    _fields_ = [("n", C.c_uint64), ("nnz", C.c_uint64), ("sum_ln", C.c_double),
+                ("sum_ln2", C.c_double), ("mu", C.c_double), ("sigma", C.c_double)]
+
+
+class FpFormatT(C.Structure):
+    _fields_ = [("nbits", C.c_int32), ("exp_bits", C.c_int32), ("man_bits", C.c_int32),
+                ("scale_exp", C.c_int32)]
+
+
+class LayerT(C.Structure):
+    _fields_ = [("g", C.c_void_p), ("out", C.c_void_p), ("n", C.c_uint64),
+                ("dt", C.c_int32), ("mode", C.c_int32), ("S", C.c_double),
+                ("nbits", C.c_int32), ("rounding", C.c_int32), ("seed", C.c_uint64),
+                ("use_override", C.c_int32), ("reserved", C.c_int32),
+                ("mu_override", C.c_double), ("sigma_override", C.c_double)]
+
+
+class LayerResultT(C.Structure):
+    _fields_ = [("stats", StatsT), ("tau", C.c_double), ("fmt", FpFormatT),
+                ("status", C.c_int32), ("reserved", C.c_int32)]
+
+
+assert C.sizeof(StatsT) == 48 and C.sizeof(LayerT) == 80 and C.sizeof(LayerResultT) == 80
+
+_vp, _u64, _sz, _dbl, _i32 = C.c_void_p, C.c_uint64, C.c_size_t, C.c_double, C.c_int
+_lib.lgn_status_string.argtypes = [_i32]
+_lib.lgn_status_string.restype = C.c_char_p
+_lib.lgn_workspace_bytes.argtypes = [C.POINTER(_u64), _i32]
+_lib.lgn_workspace_bytes.restype = _sz
+_lib.lgn_codes_bytes.argtypes = [_u64, _i32]
+_lib.lgn_codes_bytes.restype = _sz
+_lib.lgn_stats.argtypes = [_vp, _u64, _i32, _vp, _vp, _sz, _vp]
+_lib.lgn_stats.restype = _i32
+_lib.lgn_threshold.argtypes = [_dbl, _dbl, _dbl, _dbl, C.POINTER(_dbl)]
+_lib.lgn_threshold.restype = _i32
+_lib.lgn_snap_threshold.argtypes = [_dbl, _i32]
+_lib.lgn_snap_threshold.restype = _dbl
+_lib.lgn_fp_format.argtypes = [_dbl, _dbl, _i32, C.POINTER(FpFormatT)]
+_lib.lgn_fp_format.restype = _i32
+_lib.lgn_prune.argtypes = [_vp, _vp, _u64, _i32, _dbl, _u64, _vp]
+_lib.lgn_prune.restype = _i32
+_lib.lgn_quantize.argtypes = [_vp, _vp, _u64, _i32, C.POINTER(FpFormatT), _i32, _u64, _vp]
+_lib.lgn_quantize.restype = _i32
+_lib.lgn_compress_layers.argtypes = [C.POINTER(LayerT), _i32, _vp, _vp, _sz, _vp]
+_lib.lgn_compress_layers.restype = _i32
+
+
+class LgnError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {_lib.lgn_status_string(code).decode()} (status {code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != LGN_OK:
+        raise LgnError(code, where)
+
+
+def raw():
+    """The loaded ctypes library (for tests of the ABI itself)."""
+    return _lib
+
+
+def dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"gradient tensors are float32 or bfloat16, got {t.dtype}")
+
+
+def _dev(t: torch.Tensor, what: str) -> int:
+    if not t.is_cuda:
+        raise ValueError(f"{what} must be a CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{what} must be contiguous")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+# --------------------------------------------------------------------------- sizes
+def lgn_workspace_bytes(n_per_layer: Sequence[int]) -> int:
+    arr = (_u64 * max(1, len(n_per_layer)))(*n_per_layer)
+    return int(_lib.lgn_workspace_bytes(arr, len(n_per_layer)))
+
+
+def lgn_codes_bytes(n: int, nbits: int) -> int:
+    return int(_lib.lgn_codes_bytes(n, nbits))
+
+
+def new_workspace(n_per_layer: Sequence[int], device) -> torch.Tensor:
+    return torch.empty(max(16, lgn_workspace_bytes(n_per_layer)), dtype=torch.uint8, device=device)
+
+
+# --------------------------------------------------------------------------- host closed forms
+def lgn_threshold(mu: float, sigma: float, zero_frac: float, S: float) -> float:
+    tau = _dbl()
+    _check(_lib.lgn_threshold(mu, sigma, zero_frac, S, C.byref(tau)), "lgn_threshold")
+    return tau.value
+
+
+def lgn_snap_threshold(tau: float, dt: int) -> float:
+    return float(_lib.lgn_snap_threshold(tau, dt))
+
+
+def lgn_fp_format(mu: float, sigma: float, nbits: int) -> Dict[str, int]:
+    f = FpFormatT()
+    _check(_lib.lgn_fp_format(mu, sigma, nbits, C.byref(f)), "lgn_fp_format")
+    return {"nbits": f.nbits, "exp_bits": f.exp_bits, "man_bits": f.man_bits, "scale_exp": f.scale_exp}
+
+
+def _fmt_struct(fmt: Dict[str, int]) -> FpFormatT:
+    return FpFormatT(fmt["nbits"], fmt["exp_bits"], fmt["man_bits"], fmt["scale_exp"])
+
+
+# --------------------------------------------------------------------------- device entry points
+def lgn_stats_async(g: torch.Tensor, out_dev: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
+    """Enqueue the statistics pass; ``out_dev`` (>= 48 bytes, uint8, CUDA) receives one lgn_stats_t."""
+    _check(_lib.lgn_stats(_dev(g, "g"), g.numel(), dtype_code(g), _dev(out_dev, "out_dev"),
+                          _dev(ws, "ws"), ws.numel() * ws.element_size(), _stream(stream)), "lgn_stats")
+
+
+def read_stats(out_dev: torch.Tensor) -> Dict[str, float]:
+    raw_bytes = out_dev.cpu().numpy().tobytes()[:C.sizeof(StatsT)]
+    st = StatsT.from_buffer_copy(raw_bytes)
+    return {"n": st.n, "nnz": st.nnz, "sum_ln": st.sum_ln, "sum_ln2": st.sum_ln2,
+            "mu": st.mu, "sigma": st.sigma}
+
+
+def lgn_stats(g: torch.Tensor, ws: Optional[torch.Tensor] = None, stream=None) -> Dict[str, float]:
+    """Statistics of one tensor, read back to the host (synchronises)."""
+    ws = ws if ws is not None else new_workspace([g.numel()], g.device)
+    out = torch.empty(64, dtype=torch.uint8, device=g.device)
+    lgn_stats_async(g, out, ws, stream)
+    return read_stats(out)
+
+
+def lgn_prune(g: torch.Tensor, tau: float, seed: int, out: Optional[torch.Tensor] = None,
+              stream=None) -> torch.Tensor:
+    out = out if out is not None else torch.empty_like(g)
+    _check(_lib.lgn_prune(_dev(g, "g"), _dev(out, "out"), g.numel(), dtype_code(g), float(tau),
+                          int(seed), _stream(stream)), "lgn_prune")
+    return out
+
+
+def lgn_quantize(g: torch.Tensor, fmt: Dict[str, int], rounding: int, seed: int,
+                 out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Packed codes as a uint8 tensor of lgn_codes_bytes(n, nbits) bytes."""
+    if out is None:
+        out = torch.empty(max(16, lgn_codes_bytes(g.numel(), fmt["nbits"])), dtype=torch.uint8, device=g.device)
+    f = _fmt_struct(fmt)
+    _check(_lib.lgn_quantize(_dev(g, "g"), _dev(out, "codes"), g.numel(), dtype_code(g), C.byref(f),
+                             int(rounding), int(seed), _stream(stream)), "lgn_quantize")
+    return out
+
+
+def make_layer(g: torch.Tensor, out: torch.Tensor, mode: int, S: float = 0.0, nbits: int = 0,
+               rounding: int = ROUND_NEAREST, seed: int = 0, mu_override: Optional[float] = None,
+               sigma_override: Optional[float] = None) -> LayerT:
+    use = mu_override is not None and sigma_override is not None
+    return LayerT(_dev(g, "g") if g.numel() else (g.data_ptr() or None),
+                  _dev(out, "out") if out.numel() else (out.data_ptr() or None), g.numel(), dtype_code(g),
+                  mode, float(S), int(nbits), int(rounding), int(seed), 1 if use else 0, 0,
+                  float(mu_override) if use else 0.0, float(sigma_override) if use else 0.0)
+
+
+def lgn_compress_layers(layers: Sequence[LayerT], results_dev: torch.Tensor, ws: torch.Tensor,
+                        stream=None) -> None:
+    """Enqueue the grouped path.  ``results_dev``: uint8 CUDA tensor of at least
+    80 bytes per layer; ``ws``: uint8 CUDA tensor of lgn_workspace_bytes(...)."""
+    L = len(layers)
+    arr = (LayerT * max(1, L))(*layers)
+    if results_dev.numel() * results_dev.element_size() < L * C.sizeof(LayerResultT):
+        raise ValueError("results_dev too small")
+    _check(_lib.lgn_compress_layers(arr, L, _dev(results_dev, "results_dev"), _dev(ws, "ws"),
+                                    ws.numel() * ws.element_size(), _stream(stream)), "lgn_compress_layers")
+
+
+def new_results(num_layers: int, device) -> torch.Tensor:
+    return torch.zeros(max(1, num_layers) * C.sizeof(LayerResultT), dtype=torch.uint8, device=device)
+
+
+def read_results(results_dev: torch.Tensor, num_layers: int) -> List[Dict]:
+    """Host copy of the per-layer results (synchronises)."""
+    buf = results_dev.cpu().numpy().tobytes()
+    out = []
+    for k in range(num_layers):
+        r = LayerResultT.from_buffer_copy(buf[k * C.sizeof(LayerResultT):(k + 1) * C.sizeof(LayerResultT)])
+        out.append({"n": r.stats.n, "nnz": r.stats.nnz, "sum_ln": r.stats.sum_ln, "sum_ln2": r.stats.sum_ln2,
+                    "mu": r.stats.mu, "sigma": r.stats.sigma, "tau": r.tau,
+                    "fmt": {"nbits": r.fmt.nbits, "exp_bits": r.fmt.exp_bits, "man_bits": r.fmt.man_bits,
+                            "scale_exp": r.fmt.scale_exp},
+                    "status": r.status})
+    return out

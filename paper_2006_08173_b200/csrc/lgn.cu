@@ -1,0 +1,604 @@
+// Kernels and C entry points of the lognormal gradient-compression library.
+//
+// One persistent kernel runs the whole path for a list of tensors.  Work is cut
+// into tiles of kTileElems elements; tiles of all layers sit in one queue, in an
+// order the host chooses, and CTAs pop them with one atomic each:
+//
+//   statistics tile : log2|g| partial sums of the tile -> its slot in the partial
+//                     array; the CTA that completes a layer's last statistics tile
+//                     adds the layer's partials in a fixed order, evaluates the
+//                     closed form (Eq. 8 inverse or Eq. 4 argmin) in fp64 and
+//                     publishes the result with a release store
+//   apply tile      : waits (bounded) for that publication, then prunes (Eq. 5) or
+//                     quantises and packs (Eq. 1-2) the tile
+//
+// A statistics tile never waits, and a layer's statistics tiles precede its apply
+// tiles in the queue, so every wait is on work already handed to a running CTA.
+#include <cstdio>
+#include <cstring>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "lgn.h"
+#include "lgn_closed_form.cuh"
+#include "lgn_device.cuh"
+
+namespace lgn {
+
+// ------------------------------------------------------------------ workspace layout
+struct WsHeader {
+    uint32_t queue_head;
+    uint32_t error;
+    uint32_t pad[62];
+};
+static_assert(sizeof(WsHeader) == 256, "header is one 256-byte block");
+
+constexpr int32_t kModeStatsOnly = 2;
+
+struct alignas(16) LayerState {          // written by the set-up launch, then read-only
+    const void         *g;
+    void               *out;
+    uint64_t            n;
+    uint64_t            seed;
+    double              S;
+    double              mu_override, sigma_override;
+    lgn_stats_t        *stats_out;       // may be null
+    lgn_layer_result_t *result_out;      // may be null
+    uint32_t            ntiles;
+    uint32_t            partial0;        // first slot of this layer in the partial array
+    int32_t             dt, mode, nbits, rounding, use_override, pad;
+};
+static_assert(sizeof(LayerState) == 112, "LayerState layout");
+
+struct alignas(16) LayerDyn {            // zeroed by the set-up launch, written by the kernel
+    uint32_t    done;                    // statistics tiles completed
+    uint32_t    ready;                   // 1 once tau / q below are valid
+    float       tau;
+    int32_t     status;
+    QuantParams q;
+    uint32_t    pad[2];
+};
+static_assert(sizeof(LayerDyn) == 64, "LayerDyn layout");
+
+struct alignas(16) Segment {             // a run of consecutive queue items
+    uint32_t first_item;
+    uint32_t ntiles;
+    uint32_t layer;
+    uint32_t phase;                      // 0 statistics, 1 apply
+    uint32_t tile_begin;                 // first tile of the layer this run covers
+    uint32_t reverse;                    // walk the run from its last tile down
+    uint32_t pad[2];
+};
+static_assert(sizeof(Segment) == 32, "Segment layout");
+
+struct alignas(16) Partial {
+    double             s1, s2;           // sums of log2|g| and its square over the tile's nonzeros
+    unsigned long long cnt;
+    unsigned long long pad;
+};
+
+struct WsLayout {
+    size_t states, dyn, segs, partials, total;
+    uint32_t nseg_max;
+    uint64_t total_tiles;
+};
+
+static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static bool ws_layout(const uint64_t *n_per_layer, int L, WsLayout &w) {
+    if (L < 0) return false;
+    uint64_t tiles = 0;
+    for (int k = 0; k < L; ++k) {
+        if (n_per_layer[k] > (1ull << 44)) return false;
+        tiles += (n_per_layer[k] + kTileElems - 1) / kTileElems;
+    }
+    if (tiles >= (1ull << 31)) return false;
+    w.total_tiles = tiles;
+    w.nseg_max = 2u * (uint32_t)L + 2u;
+    w.states = sizeof(WsHeader);
+    w.dyn = w.states + round_up(sizeof(LayerState) * (size_t)L, 256);
+    w.segs = w.dyn + round_up(sizeof(LayerDyn) * (size_t)L, 256);
+    w.partials = w.segs + round_up(sizeof(Segment) * (size_t)w.nseg_max, 256);
+    w.total = w.partials + round_up(sizeof(Partial) * (size_t)tiles, 256);
+    return true;
+}
+
+// ------------------------------------------------------------------ set-up launch
+// Host bytes travel to the device inside the kernel parameter block: no pinned
+// staging buffer, no synchronous copy, ordered on the stream like any launch.
+constexpr int kBlobBytes = 3840;
+struct Blob { uint4 v[kBlobBytes / 16]; };
+
+__global__ void upload_kernel(const __grid_constant__ Blob blob, uint4 *dst, int nvec) {
+    for (int i = threadIdx.x; i < nvec; i += blockDim.x) dst[i] = blob.v[i];
+}
+
+// ------------------------------------------------------------------ device helpers
+__device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(uint32_t *p, uint32_t v) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
+}
+
+template <int DT>
+__device__ __noinline__ void run_stats_tile(const LayerState &L, uint32_t tile, Partial *partials, double *sm) {
+    StatsAcc acc;
+    const uint64_t base = (uint64_t)tile * kTileElems;
+    if (base + kTileElems <= L.n) stats_tile<DT, true>(L.g, base, L.n, acc);
+    else                          stats_tile<DT, false>(L.g, base, L.n, acc);
+    block_reduce(acc, sm);
+    if (threadIdx.x == 0) {
+        Partial p;
+        p.s1 = acc.s1; p.s2 = acc.s2; p.cnt = acc.cnt; p.pad = 0;
+        partials[L.partial0 + tile] = p;
+    }
+}
+
+// Adds up a layer's partials (thread t takes slots t, t+kThreads, ... in order,
+// then the fixed tree), turns them into mu, sigma, and evaluates the closed form.
+__device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn *D, const Partial *partials, double *sm) {
+    StatsAcc acc;
+    for (uint32_t t = threadIdx.x; t < L.ntiles; t += kThreads) {
+        const Partial *p = partials + L.partial0 + t;
+        acc.s1 += __ldcg(&p->s1);
+        acc.s2 += __ldcg(&p->s2);
+        acc.cnt += __ldcg(&p->cnt);
+    }
+    block_reduce(acc, sm);
+    if (threadIdx.x != 0) return;
+
+    lgn_stats_t st;
+    st.n = L.n;
+    st.nnz = acc.cnt;
+    st.sum_ln = st.sum_ln2 = st.mu = st.sigma = 0.0;
+    if (acc.cnt) {
+        const double inv = 1.0 / (double)acc.cnt;
+        const double m2 = acc.s1 * inv;                       // mean of log2|g|
+        double var = acc.s2 * inv - m2 * m2;
+        if (!(var > 0.0)) var = 0.0;
+        st.mu = m2 * kLn2;
+        st.sigma = sqrt(var) * kLn2;
+        st.sum_ln = acc.s1 * kLn2;
+        st.sum_ln2 = acc.s2 * kLn2 * kLn2;
+    }
+    if (L.stats_out) *L.stats_out = st;
+
+    const double mu = L.use_override ? L.mu_override : st.mu;
+    const double sigma = L.use_override ? L.sigma_override : st.sigma;
+    double tau_used = 0.0;
+    lgn_fp_format_t fmt;
+    fmt.nbits = fmt.exp_bits = fmt.man_bits = fmt.scale_exp = 0;
+    if (L.mode == LGN_MODE_PRUNE) {
+        const double zero_frac = 1.0 - (double)st.nnz / (double)st.n;
+        const double tau = acc.cnt ? threshold_for(mu, sigma, zero_frac, L.S) : 0.0;
+        const float t = (L.dt == LGN_BF16) ? snap_threshold_bf16(tau) : snap_threshold_f32(tau);
+        D->tau = t;
+        tau_used = (double)t;
+    } else if (L.mode == LGN_MODE_QUANTIZE) {
+        if (acc.cnt) {
+            choose_format(mu, sigma, L.nbits, fmt);
+        } else {                                              // all zero: every code is 0 anyway
+            fmt.nbits = L.nbits; fmt.exp_bits = 1; fmt.man_bits = L.nbits - 2; fmt.scale_exp = 0;
+        }
+        D->q = make_quant_params(fmt);
+    }
+    if (L.result_out) {
+        lgn_layer_result_t r;
+        r.stats = st; r.tau = tau_used; r.fmt = fmt; r.status = LGN_OK; r.reserved = 0;
+        *L.result_out = r;
+    }
+    __threadfence();
+    st_release(&D->ready, 1u);
+}
+
+template <int DT, int NBITS>
+__device__ __noinline__ void run_quant_tile_n(const void *g, void *out, uint64_t n, uint32_t tile,
+                                                 const QuantParams &q, bool sr, uint64_t seed) {
+    const uint64_t base = (uint64_t)tile * kTileElems;
+    const uint64_t total_words = (n * (uint64_t)NBITS + 31) >> 5;
+    uint32_t *codes = static_cast<uint32_t *>(out);
+    const bool full = base + kTileElems <= n;
+    if (sr) {
+        if (full) quant_tile<DT, NBITS, true, true>(g, codes, base, n, total_words, q, seed);
+        else      quant_tile<DT, NBITS, true, false>(g, codes, base, n, total_words, q, seed);
+    } else {
+        if (full) quant_tile<DT, NBITS, false, true>(g, codes, base, n, total_words, q, seed);
+        else      quant_tile<DT, NBITS, false, false>(g, codes, base, n, total_words, q, seed);
+    }
+}
+
+template <int DT>
+__device__ __forceinline__ void run_quant_tile(const void *g, void *out, uint64_t n, uint32_t tile, int nbits,
+                                               const QuantParams &q, bool sr, uint64_t seed) {
+    switch (nbits) {
+        case 4: run_quant_tile_n<DT, 4>(g, out, n, tile, q, sr, seed); break;
+        case 5: run_quant_tile_n<DT, 5>(g, out, n, tile, q, sr, seed); break;
+        case 6: run_quant_tile_n<DT, 6>(g, out, n, tile, q, sr, seed); break;
+        case 7: run_quant_tile_n<DT, 7>(g, out, n, tile, q, sr, seed); break;
+        default: run_quant_tile_n<DT, 8>(g, out, n, tile, q, sr, seed); break;
+    }
+}
+
+template <int DT>
+__device__ __noinline__ void run_prune_tile(const void *g, void *out, uint64_t n, uint32_t tile,
+                                               float tau, uint64_t seed) {
+    const uint64_t base = (uint64_t)tile * kTileElems;
+    if (base + kTileElems <= n) prune_tile<DT, true>(g, out, base, n, tau, seed);
+    else                        prune_tile<DT, false>(g, out, base, n, tau, seed);
+}
+
+// ------------------------------------------------------------------ the persistent kernel
+constexpr uint32_t kMaxPolls = 1u << 22;      // x ~0.25 us back-off: about one second
+
+__global__ void __launch_bounds__(kThreads, 4)
+compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Segment *segs,
+                int num_layers, uint32_t total_items, Partial *partials) {
+    __shared__ double sm_red[3 * kWarps];
+    __shared__ uint32_t sm_item[2];
+    __shared__ uint32_t sm_flag;
+
+    if (blockIdx.x == 0) {                       // layers with no elements have no tiles: answer here
+        for (int k = threadIdx.x; k < num_layers; k += kThreads) {
+            const LayerState &L = states[k];
+            if (L.ntiles != 0) continue;
+            lgn_stats_t st;
+            st.n = 0; st.nnz = 0; st.sum_ln = st.sum_ln2 = st.mu = st.sigma = 0.0;
+            if (L.stats_out) *L.stats_out = st;
+            if (L.result_out) {
+                lgn_layer_result_t r;
+                memset(&r, 0, sizeof r);
+                r.stats = st;
+                if (L.mode == LGN_MODE_QUANTIZE) { r.fmt.nbits = L.nbits; r.fmt.exp_bits = 1; r.fmt.man_bits = L.nbits - 2; }
+                *L.result_out = r;
+            }
+        }
+    }
+
+    uint32_t seg = 0;
+    for (uint32_t it = 0;; ++it) {
+        if (threadIdx.x == 0) sm_item[it & 1] = atomicAdd(&hdr->queue_head, 1u);
+        __syncthreads();
+        const uint32_t item = sm_item[it & 1];
+        if (item >= total_items) break;
+        while (item >= segs[seg].first_item + segs[seg].ntiles) ++seg;
+        const Segment sg = segs[seg];
+        uint32_t t = item - sg.first_item;
+        if (sg.reverse) t = sg.ntiles - 1u - t;
+        const uint32_t tile = sg.tile_begin + t;
+        const LayerState &L = states[sg.layer];
+        LayerDyn *D = dyn + sg.layer;
+
+        if (sg.phase == 0) {
+            if (L.dt == LGN_BF16) run_stats_tile<LGN_BF16>(L, tile, partials, sm_red);
+            else                  run_stats_tile<LGN_F32>(L, tile, partials, sm_red);
+            if (threadIdx.x == 0) {
+                __threadfence();                                   // the partial before the ticket
+                const uint32_t ticket = atomicAdd(&D->done, 1u);
+                sm_flag = (ticket == L.ntiles - 1u);
+            }
+            __syncthreads();
+            if (sm_flag) {
+                __threadfence();
+                finalize_layer(L, D, partials, sm_red);
+            }
+        } else {
+            if (threadIdx.x == 0) {
+                uint32_t polls = 0, ok = 1;
+                while (ld_acquire(&D->ready) == 0u) {
+                    if (++polls > kMaxPolls || *(volatile uint32_t *)&hdr->error) { ok = 0; break; }
+                    __nanosleep(200);
+                }
+                if (!ok) {
+                    atomicExch(&hdr->error, 1u);
+                    if (L.result_out) *(volatile int32_t *)&L.result_out->status = LGN_ERR_TIMEOUT;
+                }
+                sm_flag = ok;
+            }
+            __syncthreads();
+            if (sm_flag) {
+                if (L.mode == LGN_MODE_PRUNE) {
+                    const float tau = __ldcg(&D->tau);
+                    if (L.dt == LGN_BF16) run_prune_tile<LGN_BF16>(L.g, L.out, L.n, tile, tau, L.seed);
+                    else                  run_prune_tile<LGN_F32>(L.g, L.out, L.n, tile, tau, L.seed);
+                } else {
+                    QuantParams q;
+                    const uint4 *src = reinterpret_cast<const uint4 *>(&D->q);
+                    uint4 a = __ldcg(src), b = __ldcg(src + 1);
+                    uint2 c = __ldcg(reinterpret_cast<const uint2 *>(src + 2));
+                    uint32_t raw[10] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w, c.x, c.y};
+                    memcpy(&q, raw, sizeof q);
+                    const bool sr = L.rounding == LGN_ROUND_STOCHASTIC;
+                    if (L.dt == LGN_BF16) run_quant_tile<LGN_BF16>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed);
+                    else                  run_quant_tile<LGN_F32>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed);
+                }
+            }
+        }
+    }
+}
+static_assert(sizeof(QuantParams) == 40, "QuantParams is read as 10 words");
+
+// ------------------------------------------------------------------ stand-alone apply kernels
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 4)
+prune_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, float tau, uint64_t seed) {
+    for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)
+        run_prune_tile<DT>(g, out, n, tile, tau, seed);
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 4)
+quantize_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, int nbits, QuantParams q, int sr,
+                uint64_t seed) {
+    for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)
+        run_quant_tile<DT>(g, out, n, tile, nbits, q, sr != 0, seed);
+}
+
+// ------------------------------------------------------------------ host side
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int persistent_ctas() {
+    // resident CTAs of the largest kernel per SM x SM count of the current device
+    // (a property of the device and the binary: looked up once per device)
+    static int cached[64];
+    int dev = 0, sms = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+    if (dev >= 0 && dev < 64 && cached[dev] > 0) return cached[dev];
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel, kThreads, 0) != cudaSuccess) return -1;
+    if (per_sm < 1) per_sm = 1;
+    if (dev >= 0 && dev < 64) cached[dev] = sms * per_sm;
+    return sms * per_sm;
+}
+
+struct InternalLayer {
+    lgn_layer_t          d;
+    lgn_stats_t         *stats_out;
+    lgn_layer_result_t  *result_out;
+};
+
+static lgn_status check_layer(const lgn_layer_t &d) {
+    if (d.n > 0 && (d.g == nullptr || !aligned16(d.g))) return LGN_ERR_INVALID_ARG;
+    if (d.dt != LGN_F32 && d.dt != LGN_BF16) return LGN_ERR_INVALID_ARG;
+    if (d.mode == LGN_MODE_PRUNE) {
+        if (!(d.S >= 0.0 && d.S < 1.0)) return LGN_ERR_INVALID_ARG;
+    } else if (d.mode == LGN_MODE_QUANTIZE) {
+        if (d.nbits < 4 || d.nbits > 8) return LGN_ERR_UNSUPPORTED;
+        if (d.rounding != LGN_ROUND_NEAREST && d.rounding != LGN_ROUND_STOCHASTIC) return LGN_ERR_INVALID_ARG;
+    } else if (d.mode != kModeStatsOnly) {
+        return LGN_ERR_INVALID_ARG;
+    }
+    if (d.mode != kModeStatsOnly && d.n > 0) {
+        if (d.out == nullptr || !aligned16(d.out)) return LGN_ERR_INVALID_ARG;
+        const size_t in_bytes = d.n * (d.dt == LGN_BF16 ? 2u : 4u);
+        const size_t out_bytes = d.mode == LGN_MODE_PRUNE ? in_bytes : lgn_codes_bytes(d.n, d.nbits);
+        const char *a = static_cast<const char *>(d.g), *b = static_cast<const char *>(d.out);
+        if (a < b + out_bytes && b < a + in_bytes) return LGN_ERR_INVALID_ARG;    // overlap
+    }
+    if (d.use_override && !(d.sigma_override >= 0.0 && std::isfinite(d.mu_override) && std::isfinite(d.sigma_override)))
+        return LGN_ERR_INVALID_ARG;
+    return LGN_OK;
+}
+
+// Queue order: statistics of layer k+1 are placed between the statistics and the
+// apply tiles of layer k, so the closed form of layer k is evaluated while other
+// tiles stream; a layer's apply run walks its tiles from the last one read back to
+// the first, the order in which L2 still holds them.
+static void build_queue(const std::vector<LayerState> &st, std::vector<Segment> &segs, uint32_t &total_items) {
+    uint32_t item = 0;
+    auto push = [&](uint32_t layer, uint32_t phase) {
+        if (st[layer].ntiles == 0) return;
+        if (phase == 1 && st[layer].mode == kModeStatsOnly) return;
+        Segment s;
+        memset(&s, 0, sizeof s);
+        s.first_item = item; s.ntiles = st[layer].ntiles; s.layer = layer; s.phase = phase;
+        s.tile_begin = 0; s.reverse = phase;
+        segs.push_back(s);
+        item += s.ntiles;
+    };
+    const uint32_t L = (uint32_t)st.size();
+    for (uint32_t k = 0; k < L; ++k) {
+        push(k, 0);
+        if (k > 0) push(k - 1, 1);
+    }
+    if (L > 0) push(L - 1, 1);
+    total_items = item;
+}
+
+static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws, size_t ws_bytes, cudaStream_t stream) {
+    const int L = (int)layers.size();
+    if (L == 0) return LGN_OK;
+    std::vector<uint64_t> ns(L);
+    for (int k = 0; k < L; ++k) {
+        lgn_status s = check_layer(layers[k].d);
+        if (s != LGN_OK) return s;
+        ns[k] = layers[k].d.n;
+    }
+    WsLayout w;
+    if (!ws_layout(ns.data(), L, w)) return LGN_ERR_UNSUPPORTED;
+    if (ws == nullptr || !aligned16(ws)) return LGN_ERR_INVALID_ARG;
+    if (ws_bytes < w.total) return LGN_ERR_WORKSPACE;
+
+    std::vector<LayerState> st(L);
+    uint32_t partial0 = 0;
+    for (int k = 0; k < L; ++k) {
+        const lgn_layer_t &d = layers[k].d;
+        LayerState &s = st[k];
+        memset(&s, 0, sizeof s);
+        s.g = d.g; s.out = d.out; s.n = d.n; s.seed = d.seed; s.S = d.S;
+        s.mu_override = d.mu_override; s.sigma_override = d.sigma_override;
+        s.stats_out = layers[k].stats_out; s.result_out = layers[k].result_out;
+        s.ntiles = (uint32_t)((d.n + kTileElems - 1) / kTileElems);
+        s.partial0 = partial0;
+        s.dt = d.dt; s.mode = d.mode; s.nbits = d.nbits; s.rounding = d.rounding;
+        s.use_override = d.use_override ? 1 : 0;
+        partial0 += s.ntiles;
+    }
+    std::vector<Segment> segs;
+    uint32_t total_items = 0;
+    build_queue(st, segs, total_items);
+    {   // terminator so that the segment scan never runs off the table
+        Segment s;
+        memset(&s, 0, sizeof s);
+        s.first_item = total_items; s.ntiles = 0xFFFFFFFFu - total_items;
+        segs.push_back(s);
+    }
+
+    // image of [header | states | dyn (zero) | segments]
+    std::vector<unsigned char> image(w.partials, 0);
+    memcpy(image.data() + w.states, st.data(), sizeof(LayerState) * (size_t)L);
+    memcpy(image.data() + w.segs, segs.data(), sizeof(Segment) * segs.size());
+    const size_t used = w.segs + sizeof(Segment) * segs.size();
+    unsigned char *base = static_cast<unsigned char *>(ws);
+    for (size_t off = 0; off < used; off += kBlobBytes) {
+        Blob blob;
+        const size_t nb = used - off < (size_t)kBlobBytes ? used - off : (size_t)kBlobBytes;
+        memcpy(blob.v, image.data() + off, nb);             // nb is a multiple of 16
+        upload_kernel<<<1, 128, 0, stream>>>(blob, reinterpret_cast<uint4 *>(base + off), (int)(nb / 16));
+    }
+    if (cudaGetLastError() != cudaSuccess) return LGN_ERR_CUDA;
+
+    int grid = persistent_ctas();
+    if (grid < 1) return LGN_ERR_CUDA;
+    if ((uint32_t)grid > total_items) grid = (int)(total_items ? total_items : 1u);
+    compress_kernel<<<grid, kThreads, 0, stream>>>(
+        reinterpret_cast<WsHeader *>(base), reinterpret_cast<const LayerState *>(base + w.states),
+        reinterpret_cast<LayerDyn *>(base + w.dyn), reinterpret_cast<const Segment *>(base + w.segs),
+        L, total_items, reinterpret_cast<Partial *>(base + w.partials));
+    return cudaGetLastError() == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
+}
+
+}  // namespace lgn
+
+// ==================================================================== C ABI
+using namespace lgn;
+
+extern "C" const char *lgn_status_string(lgn_status s) {
+    switch (s) {
+        case LGN_OK: return "ok";
+        case LGN_ERR_INVALID_ARG: return "invalid argument";
+        case LGN_ERR_UNSUPPORTED: return "unsupported size or bit width";
+        case LGN_ERR_WORKSPACE: return "workspace too small";
+        case LGN_ERR_CUDA: return "CUDA runtime error";
+        case LGN_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+extern "C" size_t lgn_workspace_bytes(const uint64_t *n_per_layer, int num_layers) {
+    WsLayout w;
+    if (num_layers > 0 && n_per_layer == nullptr) return 0;
+    if (!ws_layout(n_per_layer, num_layers, w)) return 0;
+    return w.total;
+}
+
+extern "C" size_t lgn_codes_bytes(uint64_t n, int nbits) {
+    if (nbits < 4 || nbits > 8) return 0;
+    const uint64_t bytes = (n * (uint64_t)nbits + 7) / 8;
+    return (size_t)((bytes + 3) / 4 * 4);
+}
+
+extern "C" lgn_status lgn_stats(const void *g, uint64_t n, lgn_dtype dt, lgn_stats_t *out_dev,
+                                void *ws, size_t ws_bytes, void *stream) {
+    if (out_dev == nullptr || !aligned16(out_dev)) return LGN_ERR_INVALID_ARG;
+    InternalLayer il;
+    memset(&il, 0, sizeof il);
+    il.d.g = g; il.d.n = n; il.d.dt = dt; il.d.mode = kModeStatsOnly;
+    il.stats_out = out_dev;
+    return run_layers(std::vector<InternalLayer>(1, il), ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" lgn_status lgn_threshold(double mu, double sigma, double zero_frac, double S, double *tau) {
+    if (tau == nullptr) return LGN_ERR_INVALID_ARG;
+    *tau = 0.0;
+    if (!(S >= 0.0 && S < 1.0) || !(zero_frac >= 0.0 && zero_frac <= 1.0)) return LGN_ERR_INVALID_ARG;
+    if (!std::isfinite(mu) || !(sigma >= 0.0) || !std::isfinite(sigma)) return LGN_ERR_INVALID_ARG;
+    *tau = threshold_for(mu, sigma, zero_frac, S);
+    return LGN_OK;
+}
+
+extern "C" double lgn_snap_threshold(double tau, lgn_dtype dt) {
+    if (!(tau >= 0.0)) return NAN;
+    if (dt == LGN_F32) return (double)snap_threshold_f32(tau);
+    if (dt == LGN_BF16) return (double)snap_threshold_bf16(tau);
+    return NAN;
+}
+
+extern "C" lgn_status lgn_fp_format(double mu, double sigma, int nbits, lgn_fp_format_t *fmt) {
+    if (fmt == nullptr) return LGN_ERR_INVALID_ARG;
+    if (nbits < 4 || nbits > 8) return LGN_ERR_UNSUPPORTED;
+    if (!std::isfinite(mu) || !(sigma >= 0.0) || !std::isfinite(sigma)) return LGN_ERR_INVALID_ARG;
+    choose_format(mu, sigma, nbits, *fmt);
+    return LGN_OK;
+}
+
+static int apply_grid(uint32_t ntiles) {
+    int g = persistent_ctas();
+    if (g < 1) return -1;
+    return (uint32_t)g > ntiles ? (int)ntiles : g;
+}
+
+extern "C" lgn_status lgn_prune(const void *g, void *out, uint64_t n, lgn_dtype dt, double tau,
+                                uint64_t seed, void *stream) {
+    lgn_layer_t d;
+    memset(&d, 0, sizeof d);
+    d.g = g; d.out = out; d.n = n; d.dt = dt; d.mode = LGN_MODE_PRUNE; d.S = 0.0;
+    lgn_status s = check_layer(d);
+    if (s != LGN_OK) return s;
+    if (!(tau >= 0.0)) return LGN_ERR_INVALID_ARG;
+    if (n > (1ull << 44)) return LGN_ERR_UNSUPPORTED;
+    if (n == 0) return LGN_OK;
+    const uint32_t ntiles = (uint32_t)((n + kTileElems - 1) / kTileElems);
+    const int grid = apply_grid(ntiles);
+    if (grid < 1) return LGN_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dt == LGN_BF16) prune_kernel<LGN_BF16><<<grid, kThreads, 0, st>>>(g, out, n, ntiles, snap_threshold_bf16(tau), seed);
+    else                prune_kernel<LGN_F32><<<grid, kThreads, 0, st>>>(g, out, n, ntiles, snap_threshold_f32(tau), seed);
+    return cudaGetLastError() == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
+}
+
+extern "C" lgn_status lgn_quantize(const void *g, void *codes, uint64_t n, lgn_dtype dt,
+                                   const lgn_fp_format_t *fmt, lgn_rounding rounding,
+                                   uint64_t seed, void *stream) {
+    if (fmt == nullptr) return LGN_ERR_INVALID_ARG;
+    if (fmt->nbits < 4 || fmt->nbits > 8) return LGN_ERR_UNSUPPORTED;
+    if (fmt->exp_bits < 1 || fmt->man_bits < 0 || 1 + fmt->exp_bits + fmt->man_bits != fmt->nbits)
+        return LGN_ERR_INVALID_ARG;
+    if (fmt->scale_exp < -400 || fmt->scale_exp > 400) return LGN_ERR_INVALID_ARG;
+    lgn_layer_t d;
+    memset(&d, 0, sizeof d);
+    d.g = g; d.out = codes; d.n = n; d.dt = dt; d.mode = LGN_MODE_QUANTIZE; d.nbits = fmt->nbits;
+    d.rounding = rounding;
+    lgn_status s = check_layer(d);
+    if (s != LGN_OK) return s;
+    if (n > (1ull << 44)) return LGN_ERR_UNSUPPORTED;
+    if (n == 0) return LGN_OK;
+    const uint32_t ntiles = (uint32_t)((n + kTileElems - 1) / kTileElems);
+    const int grid = apply_grid(ntiles);
+    if (grid < 1) return LGN_ERR_CUDA;
+    const QuantParams q = make_quant_params(*fmt);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int sr = rounding == LGN_ROUND_STOCHASTIC;
+    if (dt == LGN_BF16) quantize_kernel<LGN_BF16><<<grid, kThreads, 0, st>>>(g, codes, n, ntiles, fmt->nbits, q, sr, seed);
+    else                quantize_kernel<LGN_F32><<<grid, kThreads, 0, st>>>(g, codes, n, ntiles, fmt->nbits, q, sr, seed);
+    return cudaGetLastError() == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
+}
+
+extern "C" lgn_status lgn_compress_layers(const lgn_layer_t *layers, int num_layers,
+                                          lgn_layer_result_t *results_dev,
+                                          void *ws, size_t ws_bytes, void *stream) {
+    if (num_layers < 0) return LGN_ERR_INVALID_ARG;
+    if (num_layers == 0) return LGN_OK;
+    if (layers == nullptr || results_dev == nullptr || !aligned16(results_dev)) return LGN_ERR_INVALID_ARG;
+    std::vector<InternalLayer> v((size_t)num_layers);
+    for (int k = 0; k < num_layers; ++k) {
+        if (layers[k].mode != LGN_MODE_PRUNE && layers[k].mode != LGN_MODE_QUANTIZE) return LGN_ERR_INVALID_ARG;
+        v[k].d = layers[k];
+        v[k].stats_out = nullptr;
+        v[k].result_out = results_dev + k;
+    }
+    return run_layers(v, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}

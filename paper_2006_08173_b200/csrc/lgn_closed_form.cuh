@@ -1,0 +1,130 @@
+// Closed forms of the lognormal model, usable from host and device code.
+//
+//   pruned_fraction / solve_threshold : Eq. 8 (sparsity of stochastic pruning
+//       as a function of the threshold) and its numerical inverse
+//   expected_rel_err / choose_format  : Eq. 4 and its minimiser
+//   snap_threshold_*                  : the threshold in the tensor's type
+#pragma once
+
+#include <cfloat>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+
+#include "lgn.h"
+
+#if defined(__CUDACC__)
+#define LGN_HD __host__ __device__ __forceinline__
+#else
+#define LGN_HD inline
+#endif
+
+namespace lgn {
+
+constexpr double kLn2      = 0.693147180559945309417232121458;
+constexpr double kInvSqrt2 = 0.707106781186547524400844362105;
+constexpr double kSigmaMin = 1e-6;
+constexpr double kSigmaMax = 25.0;
+
+LGN_HD double clamp_sigma(double s) {
+    if (!(s >= kSigmaMin)) s = kSigmaMin;
+    if (s > kSigmaMax) s = kSigmaMax;
+    return s;
+}
+
+LGN_HD double normal_cdf(double z) { return 0.5 * erfc(-z * kInvSqrt2); }
+
+// Eq. 8 in the variable u = ln(alpha / e^mu).  Writing Phi for the standard
+// normal CDF, the printed expression collapses to
+//     F(u) = Phi(u/s) - e^{s^2/2 - u} Phi((u - s^2)/s),
+// the CDF of s*N(0,1) + Exp(1) (ln of the magnitude minus ln of eps), whose
+// density is the subtracted term itself.  That term is evaluated as
+// exp(s^2/2 - u + ln Phi(.)) so that a huge exponential never meets a
+// vanishing Phi.
+LGN_HD void pruned_fraction(double u, double s, double &F, double &dF) {
+    double a = normal_cdf(u / s);
+    double pv = normal_cdf((u - s * s) / s);
+    double b = pv > 0.0 ? exp(0.5 * s * s - u + log(pv)) : 0.0;
+    F = a - b;
+    dF = b;
+}
+
+// Solve F(u) = Sp for u: Newton steps kept inside a shrinking bracket
+// (bisection whenever a step would leave it).  Sp in (0,1).
+LGN_HD double solve_threshold_u(double s, double Sp) {
+    double lo = -(40.0 * s + 50.0), hi = 40.0 * s + 50.0;
+    // start from the logistic approximation of the normal quantile, shifted
+    // by the mean of -ln(eps)
+    double q = Sp / (1.0 - Sp);
+    double u = (q > 0.0 && q < 1e300) ? s * log(q) * 0.5875 + 1.0 : 0.0;
+    if (!(u > lo && u < hi)) u = 0.0;
+    for (int it = 0; it < 200; ++it) {
+        double F, dF;
+        pruned_fraction(u, s, F, dF);
+        if (F < Sp) lo = u; else hi = u;
+        double un = u - (F - Sp) / dF;
+        if (!(un > lo && un < hi)) un = 0.5 * (lo + hi);
+        double step = fabs(un - u);
+        u = un;
+        if (step <= 4e-16 * fmax(1.0, fabs(u)) || !(hi > lo)) break;
+    }
+    return u;
+}
+
+// Appendix A.9 steps (1),(2) + Eq. 8: threshold for output sparsity S when a
+// fraction l of the tensor is already zero.
+LGN_HD double threshold_for(double mu, double sigma, double l, double S) {
+    if (!(l < 1.0)) return 0.0;
+    double Sp = (S - l) / (1.0 - l);
+    if (!(Sp > 0.0)) return 0.0;
+    double s = clamp_sigma(sigma);
+    return exp(mu + solve_threshold_u(s, Sp));
+}
+
+LGN_HD float snap_threshold_f32(double tau) {
+    float f = (float)tau;                       // round to nearest even
+    if (!(f <= FLT_MAX)) f = FLT_MAX;
+    return f;
+}
+
+LGN_HD float snap_threshold_bf16(double tau) {
+    float f = snap_threshold_f32(tau);
+    uint32_t w;
+    memcpy(&w, &f, 4);
+    w += 0x7FFFu + ((w >> 16) & 1u);            // round the low half away, ties to even
+    w &= 0xFFFF0000u;
+    if (w >= 0x7F800000u) w = 0x7F7F0000u;      // largest finite bfloat16
+    memcpy(&f, &w, 4);
+    return f;
+}
+
+// Eq. 4 with n1 mantissa / n2 exponent bits.  The exponent of Eq. 1 is base 2,
+// so the normal law of the derivation has standard deviation sigma/ln 2; in
+// terms of the natural-log sigma, E_max/(sigma/ln 2) = c and (sigma/ln 2) ln 2
+// = sigma.  Mantissa step 2^-n1.
+LGN_HD double expected_rel_err(double sigma, int n1, int n2) {
+    double Emax = (double)(1 << (n2 - 1));
+    double c = Emax * kLn2 / sigma;
+    double in_range = 2.0 * normal_cdf(c) - 1.0;
+    double t1 = in_range * exp2((double)-n1) / (8.0 * kLn2);
+    double ez = erfc((sigma + c) * kInvSqrt2);
+    double t2 = ez > 0.0 ? -exp((Emax - 1.0) * kLn2 + 0.5 * sigma * sigma + log(ez)) : 0.0;
+    double t3 = erfc(c * kInvSqrt2);
+    return t1 + t2 + t3;
+}
+
+LGN_HD void choose_format(double mu, double sigma, int nbits, lgn_fp_format_t &f) {
+    double s = clamp_sigma(sigma);
+    int best = 1;
+    double best_eta = expected_rel_err(s, nbits - 2, 1);
+    for (int n2 = 2; n2 <= nbits - 1; ++n2) {
+        double eta = expected_rel_err(s, nbits - 1 - n2, n2);
+        if (eta < best_eta) { best_eta = eta; best = n2; }
+    }
+    f.nbits = nbits;
+    f.exp_bits = best;
+    f.man_bits = nbits - 1 - best;
+    f.scale_exp = (int32_t)floor(mu / kLn2 + 0.5);
+}
+
+}  // namespace lgn

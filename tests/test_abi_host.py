@@ -1,0 +1,155 @@
+"""CPU-only checks of the C ABI: the library loads, exports what include/lgn.h
+declares, rejects bad arguments on the host, and its host-side closed forms
+agree with the oracle's."""
+import ctypes as C
+import math
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "lgn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(lgn_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lgn):
+    names = declared_functions()
+    assert {"lgn_stats", "lgn_threshold", "lgn_fp_format", "lgn_prune", "lgn_quantize",
+            "lgn_compress_layers"} <= set(names)
+    for name in names:
+        assert hasattr(lgn.raw(), name), name
+
+
+def test_struct_sizes_match_header(lgn):
+    assert C.sizeof(lgn.StatsT) == 48
+    assert C.sizeof(lgn.FpFormatT) == 16
+    assert C.sizeof(lgn.LayerT) == 80
+    assert C.sizeof(lgn.LayerResultT) == 80
+
+
+def test_status_strings(lgn):
+    seen = {lgn.raw().lgn_status_string(c).decode() for c in range(6)}
+    assert len(seen) == 6
+    assert lgn.raw().lgn_status_string(77).decode() == "unknown status"
+
+
+def test_sizes(lgn, oracle):
+    for nbits in range(4, 9):
+        for n in (0, 1, 3, 5, 1023, 2 ** 20 + 7, 2 ** 30):
+            assert lgn.lgn_codes_bytes(n, nbits) == oracle.packed_bytes(n, nbits)
+    assert lgn.lgn_codes_bytes(10, 3) == 0 and lgn.lgn_codes_bytes(10, 9) == 0
+    w1 = lgn.lgn_workspace_bytes([2 ** 20])
+    w2 = lgn.lgn_workspace_bytes([2 ** 30])
+    w3 = lgn.lgn_workspace_bytes([2 ** 20] * 53)
+    assert 0 < w1 < w2 and w1 < w3
+    assert w1 % 256 == 0
+    assert lgn.lgn_workspace_bytes([]) > 0
+    assert lgn.lgn_workspace_bytes([2 ** 50]) == 0           # too large: reported as 0
+
+
+@pytest.mark.parametrize("sigma", [1e-3, 0.3, 1.0, 1.5, 2.0, 3.0, 4.0, 5.5, 8.0, 25.0, 40.0])
+def test_threshold_agrees_with_oracle(lgn, oracle, sigma):
+    for mu in (-85.0, -12.0, 0.0, 3.0):
+        for l, S in [(0.0, 1e-6), (0.0, 0.5), (0.4, 0.8), (0.5, 0.85), (0.3, 0.99), (0.0, 1 - 1e-9),
+                     (0.5, 0.5), (0.6, 0.5), (1.0, 0.5), (0.0, 0.0)]:
+            a = lgn.lgn_threshold(mu, sigma, l, S)
+            b = oracle.threshold(mu, sigma, l, S)
+            assert a == pytest.approx(b, rel=2e-12, abs=0.0)
+            for dt in (lgn.F32, lgn.BF16):
+                assert lgn.lgn_snap_threshold(a, dt) == oracle.snap_tau(b, dt)
+
+
+def test_threshold_rejects_bad_arguments(lgn):
+    for args in [(0.0, 1.0, 0.0, 1.0), (0.0, 1.0, 0.0, -0.1), (0.0, 1.0, 1.5, 0.5), (0.0, 1.0, -0.1, 0.5),
+                 (float("nan"), 1.0, 0.0, 0.5), (0.0, -1.0, 0.0, 0.5), (0.0, float("inf"), 0.0, 0.5)]:
+        with pytest.raises(lgn.LgnError) as e:
+            lgn.lgn_threshold(*args)
+        assert e.value.code == 1
+    assert lgn.raw().lgn_threshold(0.0, 1.0, 0.0, 0.5, None) == 1
+    assert math.isnan(lgn.lgn_snap_threshold(-1.0, lgn.F32))
+    assert math.isnan(lgn.lgn_snap_threshold(1.0, 7))
+
+
+def test_snap_threshold_agrees_with_oracle(lgn, oracle):
+    rs = np.random.RandomState(0)
+    for tau in list(np.exp(rs.uniform(-100, 88, 500))) + [0.0, 1e39, 3.4e38, 2.0 ** -149, 2.0 ** -150, 1e-46]:
+        for dt in (lgn.F32, lgn.BF16):
+            assert lgn.lgn_snap_threshold(float(tau), dt) == oracle.snap_tau(float(tau), dt)
+
+
+def test_fp_format_agrees_with_oracle(lgn, oracle):
+    for nbits in range(4, 9):
+        for sigma in np.concatenate([np.linspace(0.05, 9.0, 180), [1e-9, 25.0, 60.0]]):
+            for mu in (-85.3, -12.0, -0.2, 0.0, 0.35, 4.0):
+                assert lgn.lgn_fp_format(mu, float(sigma), nbits) == oracle.fp_format(mu, float(sigma), 1, nbits)
+
+
+def test_fp_format_rejects_bad_arguments(lgn):
+    for nbits in (3, 9, 0, -1):
+        with pytest.raises(lgn.LgnError) as e:
+            lgn.lgn_fp_format(0.0, 1.0, nbits)
+        assert e.value.code == 2
+    with pytest.raises(lgn.LgnError):
+        lgn.lgn_fp_format(float("nan"), 1.0, 6)
+    assert lgn.raw().lgn_fp_format(0.0, 1.0, 6, None) == 1
+
+
+def test_device_entry_points_reject_bad_arguments_before_any_cuda_call(lgn):
+    """Fake, never dereferenced addresses: every call must return on the host."""
+    R = lgn.raw()
+    A, B, W = 0x10000, 0x90000, 0x200000                 # 16-byte aligned, disjoint
+    fmt = lgn.FpFormatT(6, 4, 1, -17)
+    INVALID, UNSUPPORTED, WORKSPACE = 1, 2, 3
+    # prune
+    assert R.lgn_prune(None, B, 100, 0, 1.0, 0, None) == INVALID
+    assert R.lgn_prune(A, None, 100, 0, 1.0, 0, None) == INVALID
+    assert R.lgn_prune(A + 4, B, 100, 0, 1.0, 0, None) == INVALID          # misaligned
+    assert R.lgn_prune(A, A + 64, 100, 0, 1.0, 0, None) == INVALID         # overlap
+    assert R.lgn_prune(A, B, 100, 5, 1.0, 0, None) == INVALID              # dtype
+    assert R.lgn_prune(A, B, 100, 0, -1.0, 0, None) == INVALID
+    assert R.lgn_prune(A, B, 100, 0, float("nan"), 0, None) == INVALID
+    assert R.lgn_prune(A, B, 0, 0, 1.0, 0, None) == 0                      # empty: nothing to do
+    # quantize
+    assert R.lgn_quantize(A, B, 100, 0, None, 0, 0, None) == INVALID
+    assert R.lgn_quantize(A, B, 100, 0, C.byref(lgn.FpFormatT(9, 5, 3, 0)), 0, 0, None) == UNSUPPORTED
+    assert R.lgn_quantize(A, B, 100, 0, C.byref(lgn.FpFormatT(6, 4, 2, 0)), 0, 0, None) == INVALID
+    assert R.lgn_quantize(A, B, 100, 0, C.byref(lgn.FpFormatT(6, 0, 5, 0)), 0, 0, None) == INVALID
+    assert R.lgn_quantize(A, B, 100, 0, C.byref(fmt), 3, 0, None) == INVALID
+    assert R.lgn_quantize(A, B + 2, 100, 0, C.byref(fmt), 0, 0, None) == INVALID
+    assert R.lgn_quantize(A, B, 0, 0, C.byref(fmt), 0, 0, None) == 0
+    # stats
+    ws_need = lgn.lgn_workspace_bytes([100])
+    assert R.lgn_stats(A, 100, 0, None, W, ws_need, None) == INVALID
+    assert R.lgn_stats(None, 100, 0, B, W, ws_need, None) == INVALID
+    assert R.lgn_stats(A, 100, 0, B, None, ws_need, None) == INVALID
+    assert R.lgn_stats(A, 100, 0, B, W, ws_need - 1, None) == WORKSPACE
+    assert R.lgn_stats(A, 2 ** 50, 0, B, W, 2 ** 40, None) == UNSUPPORTED
+    # grouped
+    def layer(**kw):
+        d = dict(g=A, out=B, n=100, dt=0, mode=0, S=0.8, nbits=6, rounding=0, seed=0,
+                 use_override=0, reserved=0, mu_override=0.0, sigma_override=0.0)
+        d.update(kw)
+        return lgn.LayerT(*[d[f[0]] for f in lgn.LayerT._fields_])
+    def call(l, ws_bytes=None, res=0x300000, n=1):
+        arr = (lgn.LayerT * 1)(l)
+        return R.lgn_compress_layers(arr, n, res, W, ws_need if ws_bytes is None else ws_bytes, None)
+    assert call(layer(S=1.0)) == INVALID
+    assert call(layer(S=-0.5)) == INVALID
+    assert call(layer(mode=7)) == INVALID
+    assert call(layer(mode=2)) == INVALID                  # the internal statistics-only mode is not public
+    assert call(layer(mode=1, nbits=3)) == UNSUPPORTED
+    assert call(layer(mode=1, rounding=2)) == INVALID
+    assert call(layer(out=None)) == INVALID
+    assert call(layer(g=A + 8)) == INVALID
+    assert call(layer(use_override=1, sigma_override=-1.0)) == INVALID
+    assert call(layer(use_override=1, mu_override=float("nan"), sigma_override=1.0)) == INVALID
+    assert call(layer(), ws_bytes=16) == WORKSPACE
+    assert call(layer(), res=None) == INVALID
+    assert call(layer(), n=-1) == INVALID
+    assert call(layer(), n=0) == 0
