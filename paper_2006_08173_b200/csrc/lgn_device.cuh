@@ -136,36 +136,60 @@ struct StatsAcc {            // per thread, in log2 units
     unsigned long long cnt = 0;
 };
 
-// Adds one tile to the thread's accumulators.  log2|x| in fp32; sums of at most
-// kRun elements in fp32, then fp64.
+// Adds one tile to the thread's accumulators.  y = log2|x| in fp32.  The sums
+// are taken of d = y - P, where the pivot P is the largest y in the first run
+// of this thread's elements that holds a nonzero: d stays of the order of the
+// spread of the data whatever its scale, so short fp32 runs of d and d^2 lose
+// nothing that matters, and a tensor whose magnitudes are all equal gives a
+// variance of exactly zero.  Runs go to fp64 accumulators; the pivot is taken
+// out again in fp64 at the end of the tile:
+//   sum y = sum d + c P,   sum y^2 = sum d^2 + 2 P sum d + c P^2.
 template <int DT, bool FULL>
 __device__ __forceinline__ void stats_tile(const void *g, uint64_t tile_base, uint64_t n, StatsAcc &acc) {
     constexpr int V = ElemTraits<DT>::kVec;
     constexpr int kLoads = kTileElems / (kThreads * V);   // 16 (fp32) or 8 (bf16)
     constexpr int kGroup = 4;                             // loads in flight per thread
+    constexpr int kRunVecs = 16 / V;                      // vectors per fp32 run of 16 elements
+    const float kUnset = -__int_as_float(0x7F800000);     // -inf: no nonzero seen yet
+    float P = kUnset;
+    double D1 = 0.0, D2 = 0.0;
+    unsigned long long C = 0;
     #pragma unroll 1
     for (int j0 = 0; j0 < kLoads; j0 += kGroup) {
         uint4 v[kGroup];
         #pragma unroll
         for (int j = 0; j < kGroup; ++j)
             v[j] = load_vec<DT, FULL, Ld::Keep>(g, tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * V, n);
-        float s1 = 0.f, s2 = 0.f;
-        uint32_t c = 0;
         #pragma unroll
-        for (int j = 0; j < kGroup; ++j) {
+        for (int r = 0; r < kGroup / kRunVecs; ++r) {
+            float y[16];
             #pragma unroll
-            for (int k = 0; k < V; ++k) {
-                float a = fabsf(u2f(elem_bits<DT>(v[j], k)));
-                bool nz = a != 0.f;
-                float y = nz ? lg2_approx(a) : 0.f;
-                s1 += y;
-                s2 = fmaf(y, y, s2);
+            for (int e = 0; e < 16; ++e)
+                y[e] = lg2_approx(fabsf(u2f(elem_bits<DT>(v[r * kRunVecs + e / V], e % V))));   // -inf for zero
+            if (P == kUnset) {
+                #pragma unroll
+                for (int e = 0; e < 16; ++e) P = fmaxf(P, y[e]);
+            }
+            float s1 = 0.f, s2 = 0.f;
+            uint32_t c = 0;
+            #pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                bool nz = y[e] != kUnset;
+                float d = nz ? y[e] - P : 0.f;
+                s1 += d;
+                s2 = fmaf(d, d, s2);
                 c += nz ? 1u : 0u;
             }
+            D1 += (double)s1;
+            D2 += (double)s2;
+            C += c;
         }
-        acc.s1 += (double)s1;
-        acc.s2 += (double)s2;
-        acc.cnt += c;
+    }
+    if (C) {
+        const double p = (double)P, c = (double)C;
+        acc.s1 += D1 + c * p;
+        acc.s2 += D2 + p * (2.0 * D1 + c * p);
+        acc.cnt += C;
     }
 }
 

@@ -9,7 +9,7 @@ REL_TOL = 1e-5      # mu / sigma: relative to the oracle's fp64 value
 
 
 def np_bits(t):
-    return synth.as_numpy_bits(t)
+    return synth.as_numpy_bits(t).reshape(-1)
 
 
 def oracle_layer(orc, g_np, mode, *, S=0.0, nbits=6, rounding=0, seed=0):
@@ -18,7 +18,8 @@ def oracle_layer(orc, g_np, mode, *, S=0.0, nbits=6, rounding=0, seed=0):
     st = orc.stats(g_np)
     res = {"stats": st}
     if mode == "prune":
-        tau = orc.snap_tau(orc.threshold(st["mu"], st["sigma"], st["zero_frac"], S), dt)
+        # a tensor with no nonzero entry has nothing to prune: tau = 0
+        tau = orc.snap_tau(orc.threshold(st["mu"], st["sigma"], st["zero_frac"], S), dt) if st["nnz"] else 0.0
         res["tau"] = tau
         res["out"] = orc.prune(g_np, tau, seed)
     else:
