@@ -1,0 +1,412 @@
+#!/usr/bin/env python
+"""Benchmark of the fused statistics -> closed form -> apply path.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step = one grouped call (lgn_compress_layers) over every tensor of the
+workload.  The default workload is the ResNet-18 backward pass at batch 256 in
+fp32: 20 conv-output gradient tensors, 635.8 M elements, pruned with per-layer
+sparsity.  Inputs are synthetic (seeded lognormal magnitudes with exact zeros)
+and resident in HBM before the clock starts.  With N > 1 (torchrun) every rank
+runs its own replica of the workload (its own micro-batch); there is no
+data-path exchange between ranks.
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2006_08173_b200 import synth  # noqa: E402
+
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+# algorithmic bytes per element: read for the statistics, read again for the
+# apply pass, write the result
+def bytes_per_elem(dtype_bytes: int, mode: str, nbits: int = 6) -> float:
+    return 2 * dtype_bytes + (dtype_bytes if mode == "prune" else nbits / 8.0)
+
+
+WORKLOADS = {
+    # name: (builder, dtype, mode, nbits, rounding)
+    "resnet18_bs256_fp32_prune": dict(net="resnet18", dtype="f32", mode="prune"),
+    "resnet18_bs256_fp32_fp6": dict(net="resnet18", dtype="f32", mode="quant", nbits=6, rounding=1),
+    "resnet50_bs256_bf16_fp6": dict(net="resnet50", dtype="bf16", mode="quant", nbits=6, rounding=1),
+    "resnet50_bs256_bf16_fp5": dict(net="resnet50", dtype="bf16", mode="quant", nbits=5, rounding=1),
+    "resnet50_bs256_bf16_prune": dict(net="resnet50", dtype="bf16", mode="prune"),
+}
+for _dt in ("fp32", "bf16"):
+    for _lg in (20, 24, 26, 28, 30):
+        WORKLOADS[f"flat_2p{_lg}_{_dt}_prune"] = dict(net="flat", log2n=_lg, dtype="f32" if _dt == "fp32" else "bf16",
+                                                      mode="prune")
+        WORKLOADS[f"flat_2p{_lg}_{_dt}_fp6"] = dict(net="flat", log2n=_lg, dtype="f32" if _dt == "fp32" else "bf16",
+                                                    mode="quant", nbits=6, rounding=1)
+
+
+def workload_specs(name: str, batch: int, seed: int):
+    w = WORKLOADS[name]
+    if w["net"] == "resnet18":
+        specs = synth.resnet18_prune_workload(batch, seed)
+    elif w["net"] == "resnet50":
+        specs = synth.resnet50_quant_workload(batch, seed)
+        if w["mode"] == "prune":
+            import numpy as np
+            rs = np.random.RandomState(seed + 1)
+            for s in specs:
+                s.sparsity = float(rs.choice([0.5, 0.7, 0.85, 0.9]))
+    else:
+        specs = [synth.LayerSpec("flat", 1 << w["log2n"], -12.0, 2.0, 0.5, 0.85, seed * 1000)]
+    return w, specs
+
+
+def read_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons of one GPU, sampled while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def dist_setup(n_gpus: int):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+    return world, rank, local
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+# --------------------------------------------------------------------------- reference arm = the oracle
+def oracle_sample(specs, w, budget_elems: int):
+    """The trailing layers of the workload, up to about budget_elems elements."""
+    chosen, total = [], 0
+    for s in reversed(specs):
+        if chosen and total + s.numel > budget_elems:
+            break
+        chosen.append(s)
+        total += s.numel
+    return list(reversed(chosen)), total
+
+
+def oracle_step(orc, arrays, specs, w):
+    """One pass of the whole path (statistics, closed form, apply) in the oracle."""
+    for g, s in zip(arrays, specs):
+        st = orc.stats(g)
+        dt = orc.BF16 if g.dtype.itemsize == 2 else orc.F32
+        if w["mode"] == "prune":
+            tau = orc.snap_tau(orc.threshold(st["mu"], st["sigma"], st["zero_frac"], s.sparsity), dt) if st["nnz"] else 0.0
+            orc.prune(g, tau, 1)
+        else:
+            f = orc.fp_format(st["mu"], st["sigma"], st["nnz"], w["nbits"])
+            codes = orc.quantize(g, f["exp_bits"], f["man_bits"], f["scale_exp"], w["rounding"], 1)
+            orc.pack(codes, w["nbits"])
+
+
+def run_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:      # under torchrun only rank 0 works; no process group
+        return
+    import oracle as orc
+    orc.build()
+    w, specs = workload_specs(args.workload, args.batch, 0)
+    dtype = torch.float32 if w["dtype"] == "f32" else torch.bfloat16
+    sample, total = oracle_sample(specs, w, args.ref_sample_elems)
+    arrays = [synth.as_numpy_bits(synth.lognormal_tensor(s.numel, s.mu, s.sigma, s.zero_frac, s.data_seed, dtype, "cpu"))
+              for s in sample]
+    bpe = bytes_per_elem(2 if w["dtype"] == "bf16" else 4, w["mode"], w.get("nbits", 6))
+    for _ in range(args.warmup):
+        oracle_step(orc, arrays, sample, w)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(orc, arrays, sample, w)
+    dt = (time.perf_counter() - t0) / args.steps
+    gbs = total * bpe / dt / 1e9
+    what = f"last {len(sample)} of {len(specs)} layers of {args.workload} ({total} elements) per step"
+    print(json.dumps({
+        "impl": "reference", "metric": "fused_stats_apply_algorithmic_GBps", "value": gbs, "unit": "GB/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": w["dtype"], "data": "synthetic",
+        "config": {"workload": args.workload, "elements_per_step": total, "sample": what},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": what},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# --------------------------------------------------------------------------- our arm
+def build_layers(lgn, w, specs, tensors, outs):
+    layers = []
+    for k, (g, o, s) in enumerate(zip(tensors, outs, specs)):
+        if w["mode"] == "prune":
+            layers.append(lgn.make_layer(g, o, lgn.MODE_PRUNE, S=s.sparsity, seed=1000 + k))
+        else:
+            layers.append(lgn.make_layer(g, o, lgn.MODE_QUANTIZE, nbits=w["nbits"], rounding=w["rounding"], seed=1000 + k))
+    return layers
+
+
+def run_ours(args):
+    world, rank, local = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    from paper_2006_08173_b200 import binding as lgn      # raises if liblgn.so is missing
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    w, specs = workload_specs(args.workload, args.batch, rank)
+    dtype = torch.float32 if w["dtype"] == "f32" else torch.bfloat16
+    esize = 4 if w["dtype"] == "f32" else 2
+    tensors = synth.make_layers(specs, dtype, str(dev))
+    if w["mode"] == "prune":
+        outs = [torch.empty_like(g) for g in tensors]
+    else:
+        outs = [torch.empty(max(16, lgn.lgn_codes_bytes(g.numel(), w["nbits"])), dtype=torch.uint8, device=dev)
+                for g in tensors]
+    layers = build_layers(lgn, w, specs, tensors, outs)
+    ws = lgn.new_workspace([g.numel() for g in tensors], dev)
+    res = lgn.new_results(len(tensors), dev)
+    total_elems = sum(g.numel() for g in tensors)
+    bpe = bytes_per_elem(esize, w["mode"], w.get("nbits", 6))
+    alg_bytes = total_elems * bpe
+    in_bytes = total_elems * esize
+    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
+    flush = None
+    if in_bytes <= 2 * l2_bytes:                     # small inputs: flush L2 between timed steps
+        flush = torch.empty(max(2 * l2_bytes, 256 << 20), dtype=torch.uint8, device=dev)
+
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        if flush is not None:
+            flush.fill_(1)
+        lgn.lgn_compress_layers(layers, res, ws)
+    torch.cuda.synchronize()
+    status = [r["status"] for r in lgn.read_results(res, len(tensors))]
+    if any(status):
+        raise SystemExit(f"per-layer status not ok: {status}")
+
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    barrier(world)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local) if rank == 0 else None
+    wall0 = time.perf_counter()
+    for i in range(args.steps):
+        if flush is not None:
+            flush.fill_(1)
+        starts[i].record(stream)
+        lgn.lgn_compress_layers(layers, res, ws)
+        ends[i].record(stream)
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - wall0
+    barrier(world)
+    clocks = sampler.stop() if sampler else None
+    per_step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    if flush is None:
+        total_ms = starts[0].elapsed_time(ends[-1])      # device time of exactly K back-to-back steps
+    else:
+        total_ms = sum(per_step_ms)                      # the flushes between steps are not part of the path
+    total_ms = max_over_ranks(total_ms, world, dev)
+    ms_per_step = total_ms / args.steps
+    value = world * alg_bytes / (ms_per_step * 1e-3) / 1e9
+
+    peak, peak_kind = read_peak()
+    kern_ms = statistics.mean(per_step_ms)
+    achieved = alg_bytes / (kern_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
+                "kernel": "compress_kernel", "algorithmic_bytes_per_launch": alg_bytes,
+                "best_ms": min(per_step_ms), "median_ms": statistics.median(per_step_ms)}
+    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(traffic_path) as f:
+            tr = json.load(f).get(args.workload)
+        if tr and tr.get("library_sha") == lib_sha():
+            roofline["traffic"] = tr["dram_bytes_per_launch"]
+    except Exception:
+        pass
+
+    line = {
+        "metric": "fused_stats_apply_algorithmic_GBps", "value": value, "unit": "GB/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": w["dtype"], "data": "synthetic",
+        "config": {"workload": args.workload, "layers": len(tensors), "elements_per_step_per_gpu": total_elems,
+                   "mode": w["mode"], "nbits": w.get("nbits"), "batch": args.batch,
+                   "l2": "inputs larger than L2" if flush is None else "L2 flushed between timed steps",
+                   "parallelism": f"replicas x{world}"},
+        "elements_per_s": world * total_elems / (ms_per_step * 1e-3),
+        "gpu_launches": args.steps * lgn.lgn_launches_per_call(len(tensors)),
+        "roofline": roofline,
+        "clocks": clocks,
+        "wall_s": wall,
+    }
+
+    if rank == 0 and not args.no_e2e:
+        line["e2e"] = measure_e2e(lgn, args, w, specs, tensors, dev, alg_bytes)
+    barrier(world)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = measure_cpu_baseline(args, w, specs, tensors, bpe)
+    if rank == 0:
+        print(json.dumps(line))
+
+
+def lib_sha():
+    import hashlib
+    h = hashlib.sha1()
+    for rel in ("paper_2006_08173_b200/csrc/lgn.cu", "paper_2006_08173_b200/csrc/lgn_device.cuh",
+                "paper_2006_08173_b200/csrc/lgn_closed_form.cuh"):
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
+
+
+def measure_e2e(lgn, args, w, specs, tensors, dev, alg_bytes):
+    """Same metric through lgn_compress_layers_host: inputs start in pinned host
+    memory, outputs and per-layer results end there; copies are inside the
+    timed region."""
+    host_in = [torch.empty(g.shape, dtype=g.dtype).pin_memory() for g in tensors]
+    for h, g in zip(host_in, tensors):
+        h.copy_(g)
+    if w["mode"] == "prune":
+        host_out = [torch.empty(g.shape, dtype=g.dtype).pin_memory() for g in tensors]
+    else:
+        host_out = [torch.empty(max(16, lgn.lgn_codes_bytes(g.numel(), w["nbits"])), dtype=torch.uint8).pin_memory()
+                    for g in tensors]
+    layers = []
+    for k, (hi, ho, s) in enumerate(zip(host_in, host_out, specs)):
+        if w["mode"] == "prune":
+            layers.append(lgn.make_host_layer(hi, ho, lgn.MODE_PRUNE, S=s.sparsity, seed=1000 + k))
+        else:
+            layers.append(lgn.make_host_layer(hi, ho, lgn.MODE_QUANTIZE, nbits=w["nbits"], rounding=w["rounding"],
+                                              seed=1000 + k))
+    dev_buf = torch.empty(lgn.lgn_host_staging_bytes(layers) + 256, dtype=torch.uint8, device=dev)
+    off = (-dev_buf.data_ptr()) % 256
+    dev_buf = dev_buf[off:]
+    lgn.lgn_compress_layers_host(layers, dev_buf)          # warm-up
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(args.e2e_steps):
+        lgn.lgn_compress_layers_host(layers, dev_buf)      # returns after the stream has drained
+    dt = (time.perf_counter() - t0) / args.e2e_steps
+    h2d = sum(h.numel() * h.element_size() for h in host_in)
+    d2h = sum(h.numel() * h.element_size() for h in host_out) + 80 * len(layers)
+    return {"value": alg_bytes / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "ms_per_step": dt * 1e3, "steps": args.e2e_steps,
+            "pcie_GBps": (h2d + d2h) / dt / 1e9}
+
+
+def measure_cpu_baseline(args, w, specs, tensors, bpe):
+    import oracle as orc
+    orc.build()
+    sample, total = oracle_sample(specs, w, args.cpu_sample_elems)
+    arrays = [synth.as_numpy_bits(tensors[len(specs) - len(sample) + k]) for k in range(len(sample))]
+    t0 = time.perf_counter()
+    oracle_step(orc, arrays, sample, w)
+    dt = time.perf_counter() - t0
+    return {"value": total * bpe / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "sample": f"last {len(sample)} of {len(specs)} layers ({total} elements), one pass, {dt:.1f} s",
+            "host_cores_available": len(os.sched_getaffinity(0))}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet18_bs256_fp32_prune", choices=sorted(WORKLOADS))
+    ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-elems", type=int, default=230_000_000)
+    ap.add_argument("--ref-sample-elems", type=int, default=33_000_000)
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

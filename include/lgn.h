@@ -80,6 +80,11 @@ const char *lgn_status_string(lgn_status s);
  * n_per_layer: host.  Returns 0 if num_layers < 0 or a tensor is too large. */
 size_t lgn_workspace_bytes(const uint64_t *n_per_layer, int num_layers);
 
+/* Kernel launches one lgn_compress_layers call of num_layers tensors enqueues:
+ * the set-up launches that carry the descriptors plus the one compute launch.
+ * (lgn_stats: the value for 1 layer; lgn_prune / lgn_quantize: always 1.) */
+int lgn_launches_per_call(int num_layers);
+
 /* Bytes of the packed code stream of n codes of nbits each:
  * ceil(n*nbits/8) rounded up to a multiple of 4.  0 for nbits outside 4..8. */
 size_t lgn_codes_bytes(uint64_t n, int nbits);
@@ -191,6 +196,23 @@ typedef struct {
 lgn_status lgn_compress_layers(const lgn_layer_t *layers, int num_layers,
                                lgn_layer_result_t *results_dev,
                                void *ws, size_t ws_bytes, void *stream);
+
+/* The grouped path for tensors that live in HOST memory: copies every input to
+ * the device, runs lgn_compress_layers, copies every output and the results
+ * back, and waits for the stream.  This is the end-to-end form of the call a
+ * training loop on another device (or a test harness) makes; the paper's own
+ * setting keeps the gradients on the accelerator and needs no copy.
+ *   layers        host array; g and out of each entry are HOST pointers
+ *                 (page-locked memory lets the copies run at full PCIe rate)
+ *   results_host  host array of num_layers results
+ *   dev_buf       device scratch of at least lgn_host_staging_bytes(layers,
+ *                 num_layers) bytes, 256-byte aligned; holds the device copies
+ *                 of inputs and outputs, the results and the workspace
+ * Returns after cudaStreamSynchronize(stream). */
+size_t lgn_host_staging_bytes(const lgn_layer_t *layers, int num_layers);
+lgn_status lgn_compress_layers_host(const lgn_layer_t *layers, int num_layers,
+                                    lgn_layer_result_t *results_host,
+                                    void *dev_buf, size_t dev_bytes, void *stream);
 
 #ifdef __cplusplus
 }

@@ -74,6 +74,12 @@ _lib.lgn_quantize.argtypes = [_vp, _vp, _u64, _i32, C.POINTER(FpFormatT), _i32, 
 _lib.lgn_quantize.restype = _i32
 _lib.lgn_compress_layers.argtypes = [C.POINTER(LayerT), _i32, _vp, _vp, _sz, _vp]
 _lib.lgn_compress_layers.restype = _i32
+_lib.lgn_host_staging_bytes.argtypes = [C.POINTER(LayerT), _i32]
+_lib.lgn_host_staging_bytes.restype = _sz
+_lib.lgn_compress_layers_host.argtypes = [C.POINTER(LayerT), _i32, C.POINTER(LayerResultT), _vp, _sz, _vp]
+_lib.lgn_compress_layers_host.restype = _i32
+_lib.lgn_launches_per_call.argtypes = [_i32]
+_lib.lgn_launches_per_call.restype = _i32
 
 
 class LgnError(RuntimeError):
@@ -118,6 +124,10 @@ def _stream(stream) -> int:
 def lgn_workspace_bytes(n_per_layer: Sequence[int]) -> int:
     arr = (_u64 * max(1, len(n_per_layer)))(*n_per_layer)
     return int(_lib.lgn_workspace_bytes(arr, len(n_per_layer)))
+
+
+def lgn_launches_per_call(num_layers: int) -> int:
+    return int(_lib.lgn_launches_per_call(num_layers))
 
 
 def lgn_codes_bytes(n: int, nbits: int) -> int:
@@ -228,3 +238,39 @@ def read_results(results_dev: torch.Tensor, num_layers: int) -> List[Dict]:
                             "scale_exp": r.fmt.scale_exp},
                     "status": r.status})
     return out
+
+
+# --------------------------------------------------------------------------- host-buffer form
+def _result_dict(r: LayerResultT) -> Dict:
+    return {"n": r.stats.n, "nnz": r.stats.nnz, "sum_ln": r.stats.sum_ln, "sum_ln2": r.stats.sum_ln2,
+            "mu": r.stats.mu, "sigma": r.stats.sigma, "tau": r.tau,
+            "fmt": {"nbits": r.fmt.nbits, "exp_bits": r.fmt.exp_bits, "man_bits": r.fmt.man_bits,
+                    "scale_exp": r.fmt.scale_exp},
+            "status": r.status}
+
+
+def make_host_layer(g: torch.Tensor, out: torch.Tensor, mode: int, **kw) -> LayerT:
+    """Descriptor whose g/out are HOST tensors (pinned memory recommended)."""
+    if g.is_cuda or out.is_cuda or not g.is_contiguous() or not out.is_contiguous():
+        raise ValueError("host layers take contiguous CPU tensors")
+    lay = LayerT(g.data_ptr() or None, out.data_ptr() or None, g.numel(), dtype_code(g), mode,
+                 float(kw.get("S", 0.0)), int(kw.get("nbits", 0)), int(kw.get("rounding", ROUND_NEAREST)),
+                 int(kw.get("seed", 0)), 0, 0, 0.0, 0.0)
+    return lay
+
+
+def lgn_host_staging_bytes(layers: Sequence[LayerT]) -> int:
+    arr = (LayerT * max(1, len(layers)))(*layers)
+    return int(_lib.lgn_host_staging_bytes(arr, len(layers)))
+
+
+def lgn_compress_layers_host(layers: Sequence[LayerT], dev_buf: torch.Tensor, stream=None) -> List[Dict]:
+    """Host tensors in, host tensors out; copies and the kernel run inside the
+    call, which returns when everything has landed."""
+    L = len(layers)
+    arr = (LayerT * max(1, L))(*layers)
+    res = (LayerResultT * max(1, L))()
+    _check(_lib.lgn_compress_layers_host(arr, L, res, _dev(dev_buf, "dev_buf"),
+                                         dev_buf.numel() * dev_buf.element_size(), _stream(stream)),
+           "lgn_compress_layers_host")
+    return [_result_dict(res[k]) for k in range(L)]

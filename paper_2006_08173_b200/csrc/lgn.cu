@@ -114,6 +114,12 @@ __global__ void upload_kernel(const __grid_constant__ Blob blob, uint4 *dst, int
     for (int i = threadIdx.x; i < nvec; i += blockDim.x) dst[i] = blob.v[i];
 }
 
+// The uploaded image is [header | states | dyn | segments]: it ends after the
+// segment table (at most two runs per layer plus the terminator).
+static size_t upload_bytes(const WsLayout &w, int L) {
+    return w.segs + sizeof(Segment) * (2u * (size_t)L + 1u);
+}
+
 // ------------------------------------------------------------------ device helpers
 __device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p) {
     uint32_t v;
@@ -451,7 +457,7 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
     std::vector<unsigned char> image(w.partials, 0);
     memcpy(image.data() + w.states, st.data(), sizeof(LayerState) * (size_t)L);
     memcpy(image.data() + w.segs, segs.data(), sizeof(Segment) * segs.size());
-    const size_t used = w.segs + sizeof(Segment) * segs.size();
+    const size_t used = upload_bytes(w, L);
     unsigned char *base = static_cast<unsigned char *>(ws);
     for (size_t off = 0; off < used; off += kBlobBytes) {
         Blob blob;
@@ -493,6 +499,14 @@ extern "C" size_t lgn_workspace_bytes(const uint64_t *n_per_layer, int num_layer
     if (num_layers > 0 && n_per_layer == nullptr) return 0;
     if (!ws_layout(n_per_layer, num_layers, w)) return 0;
     return w.total;
+}
+
+extern "C" int lgn_launches_per_call(int num_layers) {
+    if (num_layers <= 0) return 0;
+    std::vector<uint64_t> ns((size_t)num_layers, 1);
+    WsLayout w;
+    if (!ws_layout(ns.data(), num_layers, w)) return 0;
+    return (int)((upload_bytes(w, num_layers) + kBlobBytes - 1) / kBlobBytes) + 1;
 }
 
 extern "C" size_t lgn_codes_bytes(uint64_t n, int nbits) {
@@ -601,4 +615,77 @@ extern "C" lgn_status lgn_compress_layers(const lgn_layer_t *layers, int num_lay
         v[k].result_out = results_dev + k;
     }
     return run_layers(v, ws, ws_bytes, static_cast<cudaStream_t>(stream));
+}
+
+// ------------------------------------------------------------------ host-buffer form
+namespace {
+struct StagingPlan {
+    std::vector<size_t> in_off, out_off, in_bytes, out_bytes;
+    size_t results_off = 0, ws_off = 0, ws_bytes = 0, total = 0;
+};
+
+bool plan_staging(const lgn_layer_t *layers, int L, StagingPlan &p) {
+    size_t off = 0;
+    std::vector<uint64_t> ns((size_t)L);
+    p.in_off.resize(L); p.out_off.resize(L); p.in_bytes.resize(L); p.out_bytes.resize(L);
+    for (int k = 0; k < L; ++k) {
+        const lgn_layer_t &d = layers[k];
+        if (d.dt != LGN_F32 && d.dt != LGN_BF16) return false;
+        if (d.mode == LGN_MODE_QUANTIZE && (d.nbits < 4 || d.nbits > 8)) return false;
+        if (d.mode != LGN_MODE_QUANTIZE && d.mode != LGN_MODE_PRUNE) return false;
+        ns[k] = d.n;
+        p.in_bytes[k] = (size_t)d.n * (d.dt == LGN_BF16 ? 2u : 4u);
+        p.out_bytes[k] = d.mode == LGN_MODE_PRUNE ? p.in_bytes[k] : lgn_codes_bytes(d.n, d.nbits);
+        p.in_off[k] = off;  off += round_up(p.in_bytes[k], 256);
+        p.out_off[k] = off; off += round_up(p.out_bytes[k], 256);
+    }
+    p.results_off = off; off += round_up(sizeof(lgn_layer_result_t) * (size_t)L, 256);
+    WsLayout w;
+    if (!ws_layout(ns.data(), L, w)) return false;
+    p.ws_off = off; p.ws_bytes = w.total; off += w.total;
+    p.total = off;
+    return true;
+}
+}  // namespace
+
+extern "C" size_t lgn_host_staging_bytes(const lgn_layer_t *layers, int num_layers) {
+    if (num_layers <= 0 || layers == nullptr) return 0;
+    StagingPlan p;
+    return plan_staging(layers, num_layers, p) ? p.total : 0;
+}
+
+extern "C" lgn_status lgn_compress_layers_host(const lgn_layer_t *layers, int num_layers,
+                                               lgn_layer_result_t *results_host,
+                                               void *dev_buf, size_t dev_bytes, void *stream) {
+    if (num_layers < 0) return LGN_ERR_INVALID_ARG;
+    if (num_layers == 0) return LGN_OK;
+    if (layers == nullptr || results_host == nullptr || dev_buf == nullptr) return LGN_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(dev_buf) & 255u) != 0) return LGN_ERR_INVALID_ARG;
+    StagingPlan p;
+    if (!plan_staging(layers, num_layers, p)) return LGN_ERR_INVALID_ARG;
+    if (dev_bytes < p.total) return LGN_ERR_WORKSPACE;
+    for (int k = 0; k < num_layers; ++k)
+        if (layers[k].n > 0 && (layers[k].g == nullptr || layers[k].out == nullptr)) return LGN_ERR_INVALID_ARG;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *base = static_cast<char *>(dev_buf);
+    std::vector<lgn_layer_t> dev_layers(layers, layers + num_layers);
+    for (int k = 0; k < num_layers; ++k) {
+        dev_layers[k].g = base + p.in_off[k];
+        dev_layers[k].out = base + p.out_off[k];
+        if (p.in_bytes[k] &&
+            cudaMemcpyAsync(base + p.in_off[k], layers[k].g, p.in_bytes[k], cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return LGN_ERR_CUDA;
+    }
+    lgn_layer_result_t *res_dev = reinterpret_cast<lgn_layer_result_t *>(base + p.results_off);
+    lgn_status s = lgn_compress_layers(dev_layers.data(), num_layers, res_dev, base + p.ws_off, p.ws_bytes, stream);
+    if (s != LGN_OK) { cudaStreamSynchronize(st); return s; }
+    for (int k = 0; k < num_layers; ++k)
+        if (p.out_bytes[k] &&
+            cudaMemcpyAsync(layers[k].out, base + p.out_off[k], p.out_bytes[k], cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return LGN_ERR_CUDA;
+    if (cudaMemcpyAsync(results_host, res_dev, sizeof(lgn_layer_result_t) * (size_t)num_layers,
+                        cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return LGN_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
 }
