@@ -47,12 +47,12 @@ def _L():
         u32, u64, i32, dbl, vp = C.c_uint32, C.c_uint64, C.c_int, C.c_double, C.c_void_p
         lib.orc_stats.argtypes = [vp, u64, i32, C.POINTER(_Stats)]
         lib.orc_stats.restype = None
-        lib.orc_philox4x32_10.argtypes = [vp, vp, vp]
-        lib.orc_philox4x32_10.restype = None
-        lib.orc_rand32.argtypes = [u64, u64]
-        lib.orc_rand32.restype = u32
-        lib.orc_rand32_fill.argtypes = [u64, u64, u64, vp]
-        lib.orc_rand32_fill.restype = None
+        lib.orc_philox4x32.argtypes = [vp, vp, i32, vp]
+        lib.orc_philox4x32.restype = None
+        lib.orc_rand16.argtypes = [u64, u64]
+        lib.orc_rand16.restype = u32
+        lib.orc_rand16_fill.argtypes = [u64, u64, u64, vp]
+        lib.orc_rand16_fill.restype = None
         lib.orc_sparsity_of.argtypes = [dbl, dbl]
         lib.orc_sparsity_of.restype = dbl
         lib.orc_threshold.argtypes = [dbl, dbl, dbl, dbl, C.POINTER(dbl)]
@@ -115,21 +115,25 @@ def stats(g: np.ndarray) -> dict:
 
 
 # --------------------------------------------------------------------------- rng
-def philox4x32_10(ctr, key):
+PHILOX_ROUNDS = 7      # rounds the method uses (the known-answer vectors are for 10)
+
+
+def philox4x32(ctr, key, rounds: int = 10):
     c = np.asarray(ctr, dtype=np.uint32)
     k = np.asarray(key, dtype=np.uint32)
     o = np.zeros(4, dtype=np.uint32)
-    _L().orc_philox4x32_10(_ptr(c), _ptr(k), _ptr(o))
+    _L().orc_philox4x32(_ptr(c), _ptr(k), rounds, _ptr(o))
     return o
 
 
-def rand32(seed: int, i: int) -> int:
-    return int(_L().orc_rand32(seed, i))
+def rand16(seed: int, i: int) -> int:
+    """The 16 random bits of element i."""
+    return int(_L().orc_rand16(seed, i))
 
 
-def rand32_fill(seed: int, first: int, n: int) -> np.ndarray:
-    o = np.zeros(n, dtype=np.uint32)
-    _L().orc_rand32_fill(seed, first, n, _ptr(o))
+def rand16_fill(seed: int, first: int, n: int) -> np.ndarray:
+    o = np.zeros(n, dtype=np.uint16)
+    _L().orc_rand16_fill(seed, first, n, _ptr(o))
     return o
 
 
@@ -157,7 +161,7 @@ def prune_one(x: float, tau_used: float, h: int) -> float:
 
 def prune_with_bits(g: np.ndarray, tau_used: float, h: np.ndarray) -> np.ndarray:
     g = _flat(g)
-    h = np.ascontiguousarray(h, dtype=np.uint32)
+    h = np.ascontiguousarray(h, dtype=np.uint16)
     assert h.size == g.size
     out = np.empty_like(g)
     _L().orc_prune_with_bits(_ptr(g), _ptr(out), g.size, _dtype_of(g), tau_used, _ptr(h))
@@ -198,7 +202,7 @@ def quantize_with_bits(g, n2, n1, e_s, rounding, h=None) -> np.ndarray:
     codes = np.empty(g.size, dtype=np.uint8)
     hp = None
     if h is not None:
-        h = np.ascontiguousarray(h, dtype=np.uint32)
+        h = np.ascontiguousarray(h, dtype=np.uint16)
         assert h.size == g.size
         hp = _ptr(h)
     _L().orc_quantize_with_bits(_ptr(g), _ptr(codes), g.size, _dtype_of(g), n2, n1, e_s, rounding, hp)

@@ -23,7 +23,7 @@
  *                      Table 2 of the paper; the constants printed in the
  *                      derivation of Eq. 4; Monte-Carlo with orc_quantize
  *   orc_quantize_*     brute force over every code of every format
- *   orc_philox4x32_10  known-answer vectors published with the generator
+ *   orc_philox4x32     known-answer vectors published with the generator (10 rounds)
  *   end-to-end tensors parity unpinned by the paper (it prints no worked
  *                      numeric example of a compressed tensor)
  *
@@ -134,11 +134,11 @@ static void philox_round(uint32_t c[4], const uint32_t k[2])
     c[0] = n0; c[1] = n1; c[2] = n2; c[3] = n3;
 }
 
-void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+void orc_philox4x32(const uint32_t ctr[4], const uint32_t key[2], int rounds, uint32_t out[4])
 {
     uint32_t c[4] = { ctr[0], ctr[1], ctr[2], ctr[3] };
     uint32_t k[2] = { key[0], key[1] };
-    for (int r = 0; r < 10; ++r) {
+    for (int r = 0; r < rounds; ++r) {
         if (r) {                       /* Weyl key schedule between rounds */
             k[0] += 0x9E3779B9u;
             k[1] += 0xBB67AE85u;
@@ -148,22 +148,28 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
     memcpy(out, c, sizeof c);
 }
 
-/* The 32 random bits of element i under `seed`: key = the seed's two
- * halves, counter = (i/4 low, i/4 high, 0, 0), word i mod 4 of the block.
- * A pure function of (seed, i). */
-uint32_t orc_rand32(uint64_t seed, uint64_t i)
+/* The method draws 16 random bits per element from Philox4x32-7 (seven rounds:
+ * the fewest for which the generator's authors report a clean BigCrush run;
+ * ten is their default with a safety margin).  One 128-bit block serves the
+ * eight elements 8b..8b+7: key = the seed's two halves, counter = (b low,
+ * b high, 0, 0); element i takes word (i/2) mod 4, low half if i is even,
+ * high half if odd.  A pure function of (seed, i). */
+enum { ORC_PHILOX_ROUNDS = 7 };
+
+uint32_t orc_rand16(uint64_t seed, uint64_t i)
 {
-    uint64_t blk = i >> 2;
+    uint64_t blk = i >> 3;
     uint32_t ctr[4] = { (uint32_t)blk, (uint32_t)(blk >> 32), 0u, 0u };
     uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
     uint32_t o[4];
-    orc_philox4x32_10(ctr, key, o);
-    return o[i & 3u];
+    orc_philox4x32(ctr, key, ORC_PHILOX_ROUNDS, o);
+    uint32_t w = o[(i >> 1) & 3u];
+    return (i & 1u) ? (w >> 16) : (w & 0xFFFFu);
 }
 
-void orc_rand32_fill(uint64_t seed, uint64_t first, uint64_t n, uint32_t *out)
+void orc_rand16_fill(uint64_t seed, uint64_t first, uint64_t n, uint16_t *out)
 {
-    for (uint64_t j = 0; j < n; ++j) out[j] = orc_rand32(seed, first + j);
+    for (uint64_t j = 0; j < n; ++j) out[j] = (uint16_t)orc_rand16(seed, first + j);
 }
 
 /* ------------------------------------------------------------------ */
@@ -235,8 +241,8 @@ double orc_snap_tau(double tau, int dtype)
 /* Section 5, Eq. 5: stochastic pruning                                 */
 /* ------------------------------------------------------------------ */
 
-/* T_{alpha,eps}(x) for one element, with the element's 32 random bits h
- * given.  eps = (h >> 9) / 2^23 is uniform on [0,1) in steps of 2^-23.
+/* T_{alpha,eps}(x) for one element, with the element's 16 random bits h
+ * given.  eps = h / 2^16 is uniform on [0,1) in steps of 2^-16.
  * The product alpha*eps is rounded once to fp32 (the precision the kernel
  * compares in); |x| and alpha are exact in fp32.
  *   |x| > alpha            -> x
@@ -246,7 +252,7 @@ double orc_prune_one(double x, double tau_used, uint32_t h)
 {
     double a = fabs(x);
     if (a > tau_used) return x;
-    double eps = (double)(h >> 9) / 8388608.0;
+    double eps = (double)(h & 0xFFFFu) / 65536.0;
     double thr = (double)(float)(tau_used * eps);   /* exact product, one rounding */
     if (a != 0.0 && a >= thr) return x < 0.0 ? -tau_used : tau_used;
     return 0.0;
@@ -265,7 +271,7 @@ static void store_elem(void *out, int dtype, uint64_t i, double v)
 
 /* Whole tensor, random bits supplied by the caller (h[i] belongs to element i). */
 void orc_prune_with_bits(const void *g, void *out, uint64_t n, int dtype,
-                         double tau_used, const uint32_t *h)
+                         double tau_used, const uint16_t *h)
 {
     for (uint64_t i = 0; i < n; ++i)
         store_elem(out, dtype, i, orc_prune_one(elem(g, dtype, i), tau_used, h[i]));
@@ -278,7 +284,7 @@ void orc_prune(const void *g, void *out, uint64_t n, int dtype,
 {
     for (uint64_t i = 0; i < n; ++i)
         store_elem(out, dtype, i,
-                   orc_prune_one(elem(g, dtype, i), tau_used, orc_rand32(seed, first + i)));
+                   orc_prune_one(elem(g, dtype, i), tau_used, orc_rand16(seed, first + i)));
 }
 
 /* ------------------------------------------------------------------ */
@@ -355,16 +361,17 @@ enum { ORC_ROUND_NEAREST = 0, ORC_ROUND_STOCHASTIC = 1 };
  *                  that also has to hold zero, so the clip value is the
  *                  largest code: exponent field 2^n2 - 1, mantissa all ones.
  *   E <= -E_max -> 0 under round-to-nearest.  Under stochastic rounding the
- *                  value goes to the smallest normal 2^(1-E_max) with
- *                  probability |x'| / 2^(1-E_max) (cut to 24 bits) and to 0
- *                  otherwise: Eq. 5 with alpha = the smallest normal.
+ *                  value is pruned by Eq. 5 with alpha = the smallest normal
+ *                  (in the tensor's own units, 2^(1-E_max+e_s) as an fp32
+ *                  number) and eps = h/2^16: it becomes the smallest normal
+ *                  if |x| >= fl32(alpha*eps) and 0 otherwise, exactly as
+ *                  orc_prune_one decides.
  *   otherwise   -> M is rounded to n1 fraction bits (step Delta = 2^-n1).
- *                  Nearest: ties to even.  Stochastic: the top 23-n1 random
- *                  bits, scaled below one step, are added and the sum is
- *                  truncated.  M_q = 2 carries into E; if that reaches E_max
+ *                  Nearest: ties to even.  Stochastic: h/2^16 of one step is
+ *                  added and the sum is truncated.  M_q = 2 carries into E; if that reaches E_max
  *                  the value is clipped as above.
  * Exponent field = E + E_max in 1..2^n2-1; field 0 is zero.  Zero carries
- * sign 0.  h = the element's 32 random bits (unused for round-to-nearest). */
+ * sign 0.  h = the element's 16 random bits (unused for round-to-nearest). */
 uint32_t orc_quantize_one(double x, int n2, int n1, int e_s, int rounding, uint32_t h)
 {
     if (x == 0.0) return 0;
@@ -381,15 +388,15 @@ uint32_t orc_quantize_one(double x, int n2, int n1, int e_s, int rounding, uint3
     if (E >= Emax) return sign | top;
     if (E <= -Emax) {
         if (rounding != ORC_ROUND_STOCHASTIC) return 0;
-        double p24 = floor(ldexp(a, 24 - (1 - Emax)));   /* floor(2^24 * a / 2^(1-Emax)) */
-        return ((double)(h >> 8) < p24) ? (sign | (1u << n1)) : 0u;
+        float alpha = (float)ldexp(1.0, 1 - Emax + e_s);             /* exact, or 0 / inf out of fp32 range */
+        double eps = (double)(h & 0xFFFFu) / 65536.0;
+        double thr = (double)(float)((double)alpha * eps);
+        return (fabs(x) >= thr) ? (sign | (1u << n1)) : 0u;
     }
     double steps = (M - 1.0) * ldexp(1.0, n1);           /* exact: M has <= 23 fraction bits */
     double m;
     if (rounding == ORC_ROUND_STOCHASTIC) {
-        int d = 23 - n1;
-        double r = (double)(h >> (32 - d));
-        m = floor(steps + ldexp(r, -d));                 /* exact sum */
+        m = floor(steps + (double)(h & 0xFFFFu) / 65536.0);   /* exact sum */
     } else {
         m = nearbyint(steps);                            /* default mode: ties to even */
     }
@@ -412,7 +419,7 @@ double orc_decode(uint32_t code, int n2, int n1, int e_s)
 /* Whole tensor -> one code per byte; random bits supplied (h may be NULL for
  * round-to-nearest). */
 void orc_quantize_with_bits(const void *g, uint8_t *codes, uint64_t n, int dtype,
-                            int n2, int n1, int e_s, int rounding, const uint32_t *h)
+                            int n2, int n1, int e_s, int rounding, const uint16_t *h)
 {
     for (uint64_t i = 0; i < n; ++i)
         codes[i] = (uint8_t)orc_quantize_one(elem(g, dtype, i), n2, n1, e_s, rounding, h ? h[i] : 0u);
@@ -423,7 +430,7 @@ void orc_quantize(const void *g, uint8_t *codes, uint64_t n, int dtype,
                   int n2, int n1, int e_s, int rounding, uint64_t seed, uint64_t first)
 {
     for (uint64_t i = 0; i < n; ++i) {
-        uint32_t h = (rounding == ORC_ROUND_STOCHASTIC) ? orc_rand32(seed, first + i) : 0u;
+        uint32_t h = (rounding == ORC_ROUND_STOCHASTIC) ? orc_rand16(seed, first + i) : 0u;
         codes[i] = (uint8_t)orc_quantize_one(elem(g, dtype, i), n2, n1, e_s, rounding, h);
     }
 }

@@ -146,7 +146,7 @@ def test_every_code_of_every_format(oracle, N, n2):
     assert vals[half + 2 ** n1:] == [-v for v in grid]
     # idempotent under both roundings, any random bits
     for c in range(2 ** n1, half):
-        for rnd, h in ((RTN, 0), (SR, 0), (SR, 0xFFFFFFFF)):
+        for rnd, h in ((RTN, 0), (SR, 0), (SR, 0xFFFF)):
             assert oracle.quantize_one(vals[c], n2, n1, e_s, rnd, h) == c
             assert oracle.quantize_one(-vals[c], n2, n1, e_s, rnd, h) == c + half
     assert oracle.quantize_one(0.0, n2, n1, e_s, RTN) == 0
@@ -163,7 +163,7 @@ def test_every_code_of_every_format(oracle, N, n2):
     # clipping: everything from half a step above the largest code upward -> largest code
     top = half - 1
     for x in (grid[-1] * (1 + 2.0 ** -(n1 + 1)), grid[-1] * 2, grid[-1] * 1e6, 2.0 ** (Emax + e_s)):
-        for rnd, h in ((RTN, 0), (SR, 0), (SR, 0xFFFFFFFF)):
+        for rnd, h in ((RTN, 0), (SR, 0), (SR, 0xFFFF)):
             assert oracle.quantize_one(float(np.float32(x)), n2, n1, e_s, rnd, h) == top
     # underflow: E <= -Emax means |x| < smallest normal; nearest flushes all of it
     mn = grid[0]
@@ -189,39 +189,54 @@ def test_round_to_nearest_is_nearest_grid_point(oracle, N, n2):
 
 
 def test_stochastic_rounding_probabilities_are_exact(oracle):
-    """All 2^d values of the random field for one x: the count that rounds up
-    is exactly the dropped fraction."""
-    for (n2, n1, f) in [(4, 1, 0x2ABCDE), (5, 0, 0x000001), (3, 4, 0x7FFFFF), (2, 3, 0x400000)]:
+    """All 2^16 values of an element's random bits for one x: the count that
+    rounds up is the dropped fraction, cut to 16 bits."""
+    for (n2, n1, f) in [(4, 1, 0x2ABCDE), (5, 0, 0x000001), (5, 0, 0x000100), (3, 4, 0x7FFFFF), (2, 3, 0x400000),
+                        (4, 1, 0x3FFFFF), (4, 1, 0x400000)]:
         d = 23 - n1
         bits = np.uint32(0x3F800000 | f)                  # x in [1,2), E = 0
-        x = np.full(2 ** d, bits, dtype=np.uint32).view(np.float32)
-        h = (np.arange(2 ** d, dtype=np.uint64) << (32 - d)).astype(np.uint32)
+        x = np.full(2 ** 16, bits, dtype=np.uint32).view(np.float32)
+        h = np.arange(2 ** 16, dtype=np.uint16)
         codes = oracle.quantize_with_bits(x, n2, n1, 0, SR, h)
         lo_code = oracle.quantize_one(float(x[0]), n2, n1, 0, SR, 0)
         ups = int(np.sum(codes != lo_code))
-        assert ups == f % (2 ** d)
-        up_vals = set(np.unique(codes)) - {lo_code}
+        frac = Fraction(f % (2 ** d), 2 ** d)             # position between the two neighbours
+        assert ups == int(frac * 2 ** 16)                 # floor(frac * 2^16)
+        assert np.all(np.diff((codes != lo_code).astype(int)) >= 0)      # up exactly for the largest h
         if ups:
-            (hi_code,) = up_vals
+            (hi_code,) = set(np.unique(codes)) - {lo_code}
             step = oracle.decode(hi_code, n2, n1, 0) - oracle.decode(lo_code, n2, n1, 0)
             assert step == 2.0 ** -n1
-        # low random bits (below the field) are ignored
-        assert oracle.quantize_one(float(x[0]), n2, n1, 0, SR, (1 << (32 - d)) - 1) == lo_code
 
 
-def test_stochastic_underflow_probability(oracle):
-    n2, n1, e_s = 4, 1, 0
-    mn = 2.0 ** (1 - 8)
-    for frac in (0.3, 0.75, 2.0 ** -10, 0.999999):
-        x = float(np.float32(mn * frac))
-        p24 = int(Fraction(x) / Fraction(mn) * 2 ** 24)        # floor of the exact ratio
+def test_stochastic_underflow_is_eq5_with_the_smallest_normal(oracle):
+    """Below the smallest normal, stochastic rounding decides exactly as
+    stochastic pruning with alpha = the smallest normal does."""
+    for n2, n1, e_s in [(4, 1, 0), (5, 0, -17), (3, 2, -140), (2, 3, 5)]:
+        Emax = 2 ** (n2 - 1)
+        mn = 2.0 ** (1 - Emax + e_s)
         one = 1 << n1
-        if p24 > 0:
-            assert oracle.quantize_one(x, n2, n1, e_s, SR, ((p24 - 1) << 8) | 0xFF) == one
-            assert oracle.quantize_one(-x, n2, n1, e_s, SR, 0) == one + 32
-        assert oracle.quantize_one(x, n2, n1, e_s, SR, (p24 << 8) & 0xFFFFFFFF) == 0
-        assert oracle.quantize_one(x, n2, n1, e_s, RTN, 0) == 0
-    assert oracle.quantize_one(mn * 2.0 ** -30, n2, n1, e_s, SR, 0) == 0
+        sign = 1 << (n1 + n2)
+        rs = np.random.RandomState(n2)
+        for frac in [0.3, 0.75, 2.0 ** -10, 0.999999, 2.0 ** -17, 0.5] + list(rs.uniform(0, 1, 20)):
+            x = float(np.float32(mn * frac))
+            if x == 0.0 or x >= mn:
+                continue
+            for h in [0, 1, 0x7FFF, 0x8000, 0xFFFF] + list(rs.randint(0, 65536, 40)):
+                want = oracle.prune_one(x, float(np.float32(mn)), int(h))
+                assert want in (0.0, float(np.float32(mn)))
+                got = oracle.quantize_one(x, n2, n1, e_s, SR, int(h))
+                assert got == (one if want != 0.0 else 0)
+                assert oracle.quantize_one(-x, n2, n1, e_s, SR, int(h)) == ((one | sign) if want != 0.0 else 0)
+            assert oracle.quantize_one(x, n2, n1, e_s, RTN, 0) == 0
+        # probability of surviving = |x| / smallest normal, to 16 bits (where fp32 can
+        # resolve alpha*eps: not when the smallest normal is itself an fp32 subnormal)
+        if mn < 2.0 ** -100:
+            continue
+        x = float(np.float32(mn * 0.3))
+        hits = sum(oracle.quantize_one(x, n2, n1, e_s, SR, h) != 0 for h in range(0, 65536, 7))
+        assert abs(hits / len(range(0, 65536, 7)) - x / mn) < 2e-3
+    assert oracle.quantize_one(2.0 ** -7 * 2.0 ** -30, 4, 1, 0, SR, 1) == 0
 
 
 def test_stochastic_rounding_is_unbiased(oracle):

@@ -15,40 +15,58 @@ def test_philox_known_answers(oracle):
     assert len(rows) == 3
     for r in rows:
         w = [int(x, 16) for x in r]
-        out = oracle.philox4x32_10(w[0:4], w[4:6])
+        out = oracle.philox4x32(w[0:4], w[4:6], 10)
         assert [int(x) for x in out] == w[6:10]
 
 
-def test_rand32_is_a_pure_function_of_seed_and_index(oracle):
+def test_philox_rounds_compose(oracle):
+    """The 7-round function the method uses is the same bijection stopped
+    earlier: three more rounds, with the key advanced by seven Weyl steps, must
+    reproduce the 10-round known answers."""
+    W0, W1 = 0x9E3779B9, 0xBB67AE85
+    for r in golden_lines("philox4x32_10_kat.txt"):
+        w = [int(x, 16) for x in r]
+        mid = oracle.philox4x32(w[0:4], w[4:6], 7)
+        key7 = [(w[4] + 7 * W0) & 0xFFFFFFFF, (w[5] + 7 * W1) & 0xFFFFFFFF]
+        out = oracle.philox4x32([int(x) for x in mid], key7, 3)
+        assert [int(x) for x in out] == w[6:10]
+    assert oracle.PHILOX_ROUNDS == 7
+
+
+def test_rand16_is_a_pure_function_of_seed_and_index(oracle):
     seed = 0x1234_5678_9ABC_DEF0
-    first = (1 << 34) + 5                      # crosses the 32-bit boundary of the block counter
-    a = oracle.rand32_fill(seed, first, 64)
-    for j in (0, 1, 2, 3, 17, 63):
+    first = (1 << 35) + 5                      # crosses the 32-bit boundary of the block counter
+    a = oracle.rand16_fill(seed, first, 64)
+    for j in (0, 1, 2, 3, 10, 11, 17, 63):
         i = first + j
-        blk = i >> 2
-        ref = oracle.philox4x32_10([blk & 0xFFFFFFFF, blk >> 32, 0, 0],
-                                   [seed & 0xFFFFFFFF, seed >> 32])
-        assert int(a[j]) == int(ref[i & 3]) == oracle.rand32(seed, i)
+        blk = i >> 3
+        ref = oracle.philox4x32([blk & 0xFFFFFFFF, blk >> 32, 0, 0],
+                                [seed & 0xFFFFFFFF, seed >> 32], oracle.PHILOX_ROUNDS)
+        word = int(ref[(i >> 1) & 3])
+        want = (word >> 16) if (i & 1) else (word & 0xFFFF)
+        assert int(a[j]) == want == oracle.rand16(seed, i)
     # chunking does not matter
-    b = np.concatenate([oracle.rand32_fill(seed, first, 10), oracle.rand32_fill(seed, first + 10, 54)])
+    b = np.concatenate([oracle.rand16_fill(seed, first, 10), oracle.rand16_fill(seed, first + 10, 54)])
     assert np.array_equal(a, b)
-    assert not np.array_equal(a, oracle.rand32_fill(seed + 1, first, 64))
+    assert not np.array_equal(a, oracle.rand16_fill(seed + 1, first, 64))
 
 
-def test_rand32_uniformity(oracle):
-    n = 1 << 20
-    h = oracle.rand32_fill(1, 0, n)
-    eps = (h >> 9).astype(np.float64) / 2 ** 23
-    assert abs(eps.mean() - 0.5) < 4 * math.sqrt(1 / 12 / n)
+def test_rand16_uniformity(oracle):
+    n = 1 << 21
+    h = oracle.rand16_fill(1, 0, n).astype(np.int64)
+    eps = h / 2.0 ** 16
+    assert abs(eps.mean() - (0.5 - 2.0 ** -17)) < 4 * math.sqrt(1 / 12 / n)
     assert abs(eps.var() - 1 / 12) < 4 * math.sqrt(1 / 180 / n)
-    counts = np.bincount(h >> 24, minlength=256)
-    chi2 = ((counts - n / 256) ** 2 / (n / 256)).sum()
-    assert chi2 < 255 + 5 * math.sqrt(2 * 255)
-    lag1 = np.corrcoef(eps[:-1], eps[1:])[0, 1]
-    assert abs(lag1) < 4 / math.sqrt(n)
-    # low bits too (the stochastic-rounding field of a format with few dropped bits)
-    low = np.bincount(h & 0xFF, minlength=256)
-    assert ((low - n / 256) ** 2 / (n / 256)).sum() < 255 + 5 * math.sqrt(2 * 255)
+    for field in (h >> 8, h & 0xFF):                          # top and bottom byte
+        counts = np.bincount(field, minlength=256)
+        chi2 = ((counts - n / 256) ** 2 / (n / 256)).sum()
+        assert chi2 < 255 + 5 * math.sqrt(2 * 255)
+    for lag in (1, 2, 8):                                     # neighbours, word mates, block mates
+        c = np.corrcoef(eps[:-lag], eps[lag:])[0, 1]
+        assert abs(c) < 4 / math.sqrt(n)
+    # consecutive seeds give unrelated streams
+    g = oracle.rand16_fill(2, 0, n).astype(np.float64)
+    assert abs(np.corrcoef(eps, g)[0, 1]) < 4 / math.sqrt(n)
 
 
 # ------------------------------------------------------------------ statistics

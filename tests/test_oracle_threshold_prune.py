@@ -83,7 +83,7 @@ def test_snap_tau_matches_library_roundings(oracle):
 
 
 # ------------------------------------------------------------------ Eq. 5
-H_HALF = 0x80000000        # eps = 1/2
+H_HALF = 0x8000            # eps = 1/2 (16 random bits per element)
 
 
 def test_prune_hand_cases(oracle):
@@ -95,8 +95,8 @@ def test_prune_hand_cases(oracle):
         (-1.5, 1.0, H_HALF, -1.5),
         (0.0, 1.0, 0, 0.0),                 # eps = 0: zero still stays zero
         (1e-30, 1.0, 0, 1.0),               # eps = 0: every nonzero |x| <= alpha snaps
-        (1e-30, 1.0, 1 << 9, 0.0),          # eps = 2^-23
-        (0.999, 1.0, 0xFFFFFFFF, 0.0),      # eps = 1 - 2^-23 > 0.999
+        (1e-30, 1.0, 1, 0.0),               # eps = 2^-16
+        (0.9999, 1.0, 0xFFFF, 0.0),         # eps = 1 - 2^-16 > 0.9999
         (3.0, 0.0, H_HALF, 3.0),            # tau = 0: identity
         (0.0, 0.0, H_HALF, 0.0),
     ]
@@ -107,8 +107,8 @@ def test_prune_hand_cases(oracle):
 
 def test_prune_threshold_product_is_rounded_to_fp32(oracle):
     tau = float(np.float32(1.0 + 2 ** -23))
-    h = 0x55555555
-    eps = (h >> 9) / 2 ** 23
+    h = 0x5555
+    eps = h / 2 ** 16
     thr32 = float(np.float32(tau) * np.float32(eps))            # numpy's fp32 multiply
     exact = tau * eps
     assert thr32 != exact
@@ -138,7 +138,7 @@ def test_prune_three_value_property(oracle, dtype):
     assert np.array_equal(np.sign(y[nz]), np.sign(x[nz]))
     assert np.all(y[x == 0] == 0)
     # the seeded path is the supplied-bits path fed by the generator
-    assert np.array_equal(out, oracle.prune_with_bits(g, tau, oracle.rand32_fill(1, 0, n)))
+    assert np.array_equal(out, oracle.prune_with_bits(g, tau, oracle.rand16_fill(1, 0, n)))
     # element i depends on its global index only
     assert np.array_equal(out[1000:1300], oracle.prune(g[1000:1300], tau, seed=1, first=1000))
 
