@@ -21,8 +21,9 @@
  *    All device work is enqueued on it and the call returns without waiting.
  *  - Tensors are contiguous and are treated as flat arrays of n elements; the
  *    element index used for randomness is the flat index.
- *  - Tensor base addresses (g, out, codes, workspace, result arrays) must be
- *    16-byte aligned.  Input and output buffers must not overlap.
+ *  - Gradient tensors (g, and out of a pruning call) must be 32-byte aligned;
+ *    code streams, workspaces and result arrays 16-byte aligned.  Input and
+ *    output buffers must not overlap.
  *  - Inputs must be finite.  +0 and -0 both count as zero.
  *  - Argument errors are found on the host and returned before anything is
  *    enqueued.  A CUDA error at enqueue time is returned as LGN_ERR_CUDA.
@@ -129,9 +130,9 @@ lgn_status lgn_fp_format(double mu, double sigma, int nbits, lgn_fp_format_t *fm
  * between refreshes of the statistics.
  *   g, out  device, n elements of dt; out has the same type and layout
  *   tau     alpha >= 0; the kernel uses lgn_snap_threshold(tau, dt)
- *   seed    element i draws eps_i = (r_i >> 9) / 2^23 where r_i is word i mod 4 of
- *           Philox4x32-10 with key = (seed low, seed high), counter = (i/4 low,
- *           i/4 high, 0, 0)
+ *   seed    element i draws eps_i = h_i / 2^16, h_i = 16 bits of a Philox4x32-7
+ *           block: key = (seed low, seed high), counter = (i/8 low, i/8 high, 0, 0),
+ *           word (i/2) mod 4, low half for even i, high half for odd i
  * |g_i| > alpha -> g_i;  fl32(alpha*eps_i) <= |g_i| <= alpha -> sign(g_i)*alpha;
  * otherwise +0.  Zeros stay +0. */
 lgn_status lgn_prune(const void *g, void *out, uint64_t n, lgn_dtype dt, double tau,
@@ -146,10 +147,11 @@ lgn_status lgn_prune(const void *g, void *out, uint64_t n, lgn_dtype dt, double 
  *   seed   as in lgn_prune; used only with LGN_ROUND_STOCHASTIC
  * With x' = x / 2^scale_exp = M * 2^E, E_max = 2^(exp_bits-1):
  *   E >= E_max  (before rounding) -> largest code;
- *   E <= -E_max (before rounding) -> 0 (nearest) or, stochastic, the smallest
- *                normal with probability floor(2^24 |x'| / 2^(1-E_max)) / 2^24;
+ *   E <= -E_max (before rounding) -> 0 (nearest) or, stochastic, pruned by Eq. 5
+ *                with alpha = the smallest normal 2^(1-E_max+scale_exp) and the same
+ *                eps_i: the smallest normal if |x| >= fl32(alpha*eps_i), else 0;
  *   else M rounded to man_bits (nearest: ties to the even mantissa; stochastic:
- *   top 23-man_bits bits of r_i added below the kept bits, then truncated),
+ *   h_i/2^16 of one mantissa step added, then truncated),
  *   a carry out of M moves to E, and E reaching E_max gives the largest code.
  * Exponent field = E + E_max (1..2^exp_bits-1); field 0 encodes zero.
  * A code decodes to (-1)^s (1 + m/2^man_bits) 2^(field - E_max + scale_exp). */

@@ -57,9 +57,8 @@ struct alignas(16) LayerDyn {            // zeroed by the set-up launch, written
     float       tau;
     int32_t     status;
     QuantParams q;
-    uint32_t    pad[2];
 };
-static_assert(sizeof(LayerDyn) == 64, "LayerDyn layout");
+static_assert(sizeof(LayerDyn) == 80, "LayerDyn layout");
 
 struct alignas(16) Segment {             // a run of consecutive queue items
     uint32_t first_item;
@@ -130,18 +129,77 @@ __device__ __forceinline__ void st_release(uint32_t *p, uint32_t v) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
 }
 
+// ------------------------------------------------------------------ tile runners
+// Every pass has one hot body (whole tile inside the tensor; for quantisation
+// also the fast code path) that specialised kernels inline, and one general body
+// (ragged last tile, any layer scale) kept out of line so that it costs the hot
+// path no registers.
 template <int DT>
-__device__ __noinline__ void run_stats_tile(const LayerState &L, uint32_t tile, Partial *partials, double *sm) {
+__device__ __noinline__ void stats_tile_general(const void *g, uint64_t base, uint64_t n, StatsAcc &acc) {
+    stats_tile<DT, false>(g, base, n, acc);
+}
+
+template <int DT, bool INLINE_HOT>
+__device__ __forceinline__ void run_stats_tile(const LayerState &L, uint32_t tile, Partial *partials, double *sm) {
     StatsAcc acc;
     const uint64_t base = (uint64_t)tile * kTileElems;
-    if (base + kTileElems <= L.n) stats_tile<DT, true>(L.g, base, L.n, acc);
-    else                          stats_tile<DT, false>(L.g, base, L.n, acc);
+    if (INLINE_HOT && base + kTileElems <= L.n) stats_tile<DT, true>(L.g, base, L.n, acc);
+    else                                        stats_tile_general<DT>(L.g, base, L.n, acc);
     block_reduce(acc, sm);
     if (threadIdx.x == 0) {
         Partial p;
         p.s1 = acc.s1; p.s2 = acc.s2; p.cnt = acc.cnt; p.pad = 0;
         partials[L.partial0 + tile] = p;
     }
+}
+
+template <int DT>
+__device__ __noinline__ void prune_tile_general(const void *g, void *out, uint64_t base, uint64_t n,
+                                                float tau, uint64_t seed) {
+    prune_tile<DT, false>(g, out, base, n, tau, seed);
+}
+
+template <int DT, bool INLINE_HOT>
+__device__ __forceinline__ void run_prune_tile(const void *g, void *out, uint64_t n, uint32_t tile,
+                                               float tau, uint64_t seed) {
+    const uint64_t base = (uint64_t)tile * kTileElems;
+    if (INLINE_HOT && base + kTileElems <= n) prune_tile<DT, true>(g, out, base, n, tau, seed);
+    else                                      prune_tile_general<DT>(g, out, base, n, tau, seed);
+}
+
+template <int DT, int NBITS, bool SR>
+__device__ __noinline__ void quant_tile_general(const void *g, uint32_t *codes, uint64_t base, uint64_t n,
+                                                uint64_t total_words, const QuantParams &q, uint64_t seed) {
+    quant_tile<DT, NBITS, SR, false, false>(g, codes, base, n, total_words, q, seed);
+}
+
+template <int DT, int NBITS, bool SR, bool INLINE_HOT>
+__device__ __forceinline__ void run_quant_tile(const void *g, void *out, uint64_t n, uint32_t tile,
+                                               const QuantParams &q, uint64_t seed) {
+    const uint64_t base = (uint64_t)tile * kTileElems;
+    const uint64_t total_words = (n * (uint64_t)NBITS + 31) >> 5;
+    uint32_t *codes = static_cast<uint32_t *>(out);
+    if (INLINE_HOT && base + kTileElems <= n && q.K >= 1)
+        quant_tile<DT, NBITS, SR, true, true>(g, codes, base, n, total_words, q, seed);
+    else
+        quant_tile_general<DT, NBITS, SR>(g, codes, base, n, total_words, q, seed);
+}
+
+// run-time dispatch for groups whose layers differ in type, mode or width
+template <int DT>
+__device__ __forceinline__ void run_quant_tile_any(const void *g, void *out, uint64_t n, uint32_t tile, int nbits,
+                                                   const QuantParams &q, bool sr, uint64_t seed) {
+    #define LGN_Q(NB) \
+        if (sr) run_quant_tile<DT, NB, true, false>(g, out, n, tile, q, seed); \
+        else    run_quant_tile<DT, NB, false, false>(g, out, n, tile, q, seed);
+    switch (nbits) {
+        case 4: LGN_Q(4) break;
+        case 5: LGN_Q(5) break;
+        case 6: LGN_Q(6) break;
+        case 7: LGN_Q(7) break;
+        default: LGN_Q(8) break;
+    }
+    #undef LGN_Q
 }
 
 // Adds up a layer's partials (thread t takes slots t, t+kThreads, ... in order,
@@ -201,51 +259,30 @@ __device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn *D, co
     st_release(&D->ready, 1u);
 }
 
-template <int DT, int NBITS>
-__device__ __noinline__ void run_quant_tile_n(const void *g, void *out, uint64_t n, uint32_t tile,
-                                                 const QuantParams &q, bool sr, uint64_t seed) {
-    const uint64_t base = (uint64_t)tile * kTileElems;
-    const uint64_t total_words = (n * (uint64_t)NBITS + 31) >> 5;
-    uint32_t *codes = static_cast<uint32_t *>(out);
-    const bool full = base + kTileElems <= n;
-    if (sr) {
-        if (full) quant_tile<DT, NBITS, true, true>(g, codes, base, n, total_words, q, seed);
-        else      quant_tile<DT, NBITS, true, false>(g, codes, base, n, total_words, q, seed);
-    } else {
-        if (full) quant_tile<DT, NBITS, false, true>(g, codes, base, n, total_words, q, seed);
-        else      quant_tile<DT, NBITS, false, false>(g, codes, base, n, total_words, q, seed);
-    }
-}
-
-template <int DT>
-__device__ __forceinline__ void run_quant_tile(const void *g, void *out, uint64_t n, uint32_t tile, int nbits,
-                                               const QuantParams &q, bool sr, uint64_t seed) {
-    switch (nbits) {
-        case 4: run_quant_tile_n<DT, 4>(g, out, n, tile, q, sr, seed); break;
-        case 5: run_quant_tile_n<DT, 5>(g, out, n, tile, q, sr, seed); break;
-        case 6: run_quant_tile_n<DT, 6>(g, out, n, tile, q, sr, seed); break;
-        case 7: run_quant_tile_n<DT, 7>(g, out, n, tile, q, sr, seed); break;
-        default: run_quant_tile_n<DT, 8>(g, out, n, tile, q, sr, seed); break;
-    }
-}
-
-template <int DT>
-__device__ __noinline__ void run_prune_tile(const void *g, void *out, uint64_t n, uint32_t tile,
-                                               float tau, uint64_t seed) {
-    const uint64_t base = (uint64_t)tile * kTileElems;
-    if (base + kTileElems <= n) prune_tile<DT, true>(g, out, base, n, tau, seed);
-    else                        prune_tile<DT, false>(g, out, base, n, tau, seed);
+__device__ __forceinline__ QuantParams load_quant_params(const LayerDyn *D) {
+    const uint4 *src = reinterpret_cast<const uint4 *>(&D->q);   // written by another CTA: read through L2
+    const uint4 a = __ldcg(src), b = __ldcg(src + 1), c = __ldcg(src + 2), d = __ldcg(src + 3);
+    const uint32_t raw[16] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w, c.x, c.y, c.z, c.w, d.x, d.y, d.z, d.w};
+    QuantParams q;
+    memcpy(&q, raw, sizeof q);
+    return q;
 }
 
 // ------------------------------------------------------------------ the persistent kernel
 constexpr uint32_t kMaxPolls = 1u << 22;      // x ~0.25 us back-off: about one second
+constexpr int kAny = -1;                      // template value: decided per layer at run time
 
+// DT, MODE, NBITS, SR fix what every layer of the group has in common, so that
+// the hot tile bodies are inlined and nothing else is compiled into the kernel;
+// kAny for all four is the general kernel for mixed groups.
+template <int DT, int MODE, int NBITS, int SR>
 __global__ void __launch_bounds__(kThreads, 4)
 compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Segment *segs,
                 int num_layers, uint32_t total_items, Partial *partials) {
     __shared__ double sm_red[3 * kWarps];
     __shared__ uint32_t sm_item[2];
     __shared__ uint32_t sm_flag;
+    constexpr bool kSpecial = DT != kAny;
 
     if (blockIdx.x == 0) {                       // layers with no elements have no tiles: answer here
         for (int k = threadIdx.x; k < num_layers; k += kThreads) {
@@ -279,8 +316,12 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
         LayerDyn *D = dyn + sg.layer;
 
         if (sg.phase == 0) {
-            if (L.dt == LGN_BF16) run_stats_tile<LGN_BF16>(L, tile, partials, sm_red);
-            else                  run_stats_tile<LGN_F32>(L, tile, partials, sm_red);
+            if constexpr (kSpecial) {
+                run_stats_tile<DT, true>(L, tile, partials, sm_red);
+            } else {
+                if (L.dt == LGN_BF16) run_stats_tile<LGN_BF16, false>(L, tile, partials, sm_red);
+                else                  run_stats_tile<LGN_F32, false>(L, tile, partials, sm_red);
+            }
             if (threadIdx.x == 0) {
                 __threadfence();                                   // the partial before the ticket
                 const uint32_t ticket = atomicAdd(&D->done, 1u);
@@ -306,57 +347,86 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
             }
             __syncthreads();
             if (sm_flag) {
-                if (L.mode == LGN_MODE_PRUNE) {
-                    const float tau = __ldcg(&D->tau);
-                    if (L.dt == LGN_BF16) run_prune_tile<LGN_BF16>(L.g, L.out, L.n, tile, tau, L.seed);
-                    else                  run_prune_tile<LGN_F32>(L.g, L.out, L.n, tile, tau, L.seed);
-                } else {
-                    QuantParams q;
-                    const uint4 *src = reinterpret_cast<const uint4 *>(&D->q);
-                    uint4 a = __ldcg(src), b = __ldcg(src + 1);
-                    uint2 c = __ldcg(reinterpret_cast<const uint2 *>(src + 2));
-                    uint32_t raw[10] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w, c.x, c.y};
-                    memcpy(&q, raw, sizeof q);
-                    const bool sr = L.rounding == LGN_ROUND_STOCHASTIC;
-                    if (L.dt == LGN_BF16) run_quant_tile<LGN_BF16>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed);
-                    else                  run_quant_tile<LGN_F32>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed);
+                if constexpr (kSpecial && MODE == LGN_MODE_PRUNE) {
+                    run_prune_tile<DT, true>(L.g, L.out, L.n, tile, __ldcg(&D->tau), L.seed);
+                } else if constexpr (kSpecial && MODE == LGN_MODE_QUANTIZE) {
+                    const QuantParams q = load_quant_params(D);
+                    run_quant_tile<DT, NBITS, SR != 0, true>(L.g, L.out, L.n, tile, q, L.seed);
+                } else if constexpr (!kSpecial) {
+                    if (L.mode == LGN_MODE_PRUNE) {
+                        const float tau = __ldcg(&D->tau);
+                        if (L.dt == LGN_BF16) run_prune_tile<LGN_BF16, false>(L.g, L.out, L.n, tile, tau, L.seed);
+                        else                  run_prune_tile<LGN_F32, false>(L.g, L.out, L.n, tile, tau, L.seed);
+                    } else {
+                        const QuantParams q = load_quant_params(D);
+                        const bool sr = L.rounding == LGN_ROUND_STOCHASTIC;
+                        if (L.dt == LGN_BF16) run_quant_tile_any<LGN_BF16>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed);
+                        else                  run_quant_tile_any<LGN_F32>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed);
+                    }
                 }
             }
         }
     }
 }
-static_assert(sizeof(QuantParams) == 40, "QuantParams is read as 10 words");
 
 // ------------------------------------------------------------------ stand-alone apply kernels
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 4)
 prune_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, float tau, uint64_t seed) {
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)
-        run_prune_tile<DT>(g, out, n, tile, tau, seed);
+        run_prune_tile<DT, true>(g, out, n, tile, tau, seed);
 }
 
-template <int DT>
+template <int DT, int NBITS, int SR>
 __global__ void __launch_bounds__(kThreads, 4)
-quantize_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, int nbits, QuantParams q, int sr,
+quantize_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, const __grid_constant__ QuantParams q,
                 uint64_t seed) {
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)
-        run_quant_tile<DT>(g, out, n, tile, nbits, q, sr != 0, seed);
+        run_quant_tile<DT, NBITS, SR != 0, true>(g, out, n, tile, q, seed);
+}
+
+// ------------------------------------------------------------------ kernel tables
+// variant index: 0 statistics only, 1 prune, 2 + 2*(nbits-4) + sr quantise
+constexpr int kVariants = 12;
+#define LGN_CK(DT, MODE, NB, SR) reinterpret_cast<const void *>(&compress_kernel<DT, MODE, NB, SR>)
+#define LGN_CK_ROW(DT) { LGN_CK(DT, kModeStatsOnly, kAny, kAny), LGN_CK(DT, LGN_MODE_PRUNE, kAny, kAny), \
+    LGN_CK(DT, LGN_MODE_QUANTIZE, 4, 0), LGN_CK(DT, LGN_MODE_QUANTIZE, 4, 1), \
+    LGN_CK(DT, LGN_MODE_QUANTIZE, 5, 0), LGN_CK(DT, LGN_MODE_QUANTIZE, 5, 1), \
+    LGN_CK(DT, LGN_MODE_QUANTIZE, 6, 0), LGN_CK(DT, LGN_MODE_QUANTIZE, 6, 1), \
+    LGN_CK(DT, LGN_MODE_QUANTIZE, 7, 0), LGN_CK(DT, LGN_MODE_QUANTIZE, 7, 1), \
+    LGN_CK(DT, LGN_MODE_QUANTIZE, 8, 0), LGN_CK(DT, LGN_MODE_QUANTIZE, 8, 1) }
+static const void *const kCompressTable[2][kVariants] = { LGN_CK_ROW(LGN_F32), LGN_CK_ROW(LGN_BF16) };
+static const void *const kCompressGeneral = LGN_CK(kAny, kAny, kAny, kAny);
+#undef LGN_CK_ROW
+#undef LGN_CK
+
+#define LGN_QK(DT, NB, SR) reinterpret_cast<const void *>(&quantize_kernel<DT, NB, SR>)
+#define LGN_QK_ROW(DT) { LGN_QK(DT, 4, 0), LGN_QK(DT, 4, 1), LGN_QK(DT, 5, 0), LGN_QK(DT, 5, 1), LGN_QK(DT, 6, 0), \
+    LGN_QK(DT, 6, 1), LGN_QK(DT, 7, 0), LGN_QK(DT, 7, 1), LGN_QK(DT, 8, 0), LGN_QK(DT, 8, 1) }
+static const void *const kQuantizeTable[2][10] = { LGN_QK_ROW(LGN_F32), LGN_QK_ROW(LGN_BF16) };
+#undef LGN_QK_ROW
+#undef LGN_QK
+static const void *const kPruneTable[2] = { reinterpret_cast<const void *>(&prune_kernel<LGN_F32>),
+                                            reinterpret_cast<const void *>(&prune_kernel<LGN_BF16>) };
+
+static int variant_of(int mode, int nbits, int rounding) {
+    if (mode == kModeStatsOnly) return 0;
+    if (mode == LGN_MODE_PRUNE) return 1;
+    return 2 + 2 * (nbits - 4) + (rounding == LGN_ROUND_STOCHASTIC ? 1 : 0);
 }
 
 // ------------------------------------------------------------------ host side
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static bool aligned32(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
 
-static int persistent_ctas() {
-    // resident CTAs of the largest kernel per SM x SM count of the current device
-    // (a property of the device and the binary: looked up once per device)
-    static int cached[64];
+// Resident CTAs of `fn` per SM x SM count of the current device: the size of a
+// persistent grid.  A property of the device and the binary.
+static int persistent_ctas(const void *fn) {
     int dev = 0, sms = 0, per_sm = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return -1;
-    if (dev >= 0 && dev < 64 && cached[dev] > 0) return cached[dev];
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, compress_kernel, kThreads, 0) != cudaSuccess) return -1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, 0) != cudaSuccess) return -1;
     if (per_sm < 1) per_sm = 1;
-    if (dev >= 0 && dev < 64) cached[dev] = sms * per_sm;
     return sms * per_sm;
 }
 
@@ -367,7 +437,7 @@ struct InternalLayer {
 };
 
 static lgn_status check_layer(const lgn_layer_t &d) {
-    if (d.n > 0 && (d.g == nullptr || !aligned16(d.g))) return LGN_ERR_INVALID_ARG;
+    if (d.n > 0 && (d.g == nullptr || !aligned32(d.g))) return LGN_ERR_INVALID_ARG;
     if (d.dt != LGN_F32 && d.dt != LGN_BF16) return LGN_ERR_INVALID_ARG;
     if (d.mode == LGN_MODE_PRUNE) {
         if (!(d.S >= 0.0 && d.S < 1.0)) return LGN_ERR_INVALID_ARG;
@@ -378,7 +448,8 @@ static lgn_status check_layer(const lgn_layer_t &d) {
         return LGN_ERR_INVALID_ARG;
     }
     if (d.mode != kModeStatsOnly && d.n > 0) {
-        if (d.out == nullptr || !aligned16(d.out)) return LGN_ERR_INVALID_ARG;
+        if (d.out == nullptr || !(d.mode == LGN_MODE_PRUNE ? aligned32(d.out) : aligned16(d.out)))
+            return LGN_ERR_INVALID_ARG;
         const size_t in_bytes = d.n * (d.dt == LGN_BF16 ? 2u : 4u);
         const size_t out_bytes = d.mode == LGN_MODE_PRUNE ? in_bytes : lgn_codes_bytes(d.n, d.nbits);
         const char *a = static_cast<const char *>(d.g), *b = static_cast<const char *>(d.out);
@@ -467,13 +538,24 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
     }
     if (cudaGetLastError() != cudaSuccess) return LGN_ERR_CUDA;
 
-    int grid = persistent_ctas();
+    // one kernel per (type, mode, width, rounding) shared by all layers; the general one otherwise
+    const void *fn = kCompressTable[st[0].dt][variant_of(st[0].mode, st[0].nbits, st[0].rounding)];
+    for (int k = 1; k < L; ++k)
+        if (st[k].dt != st[0].dt || variant_of(st[k].mode, st[k].nbits, st[k].rounding) !=
+                                        variant_of(st[0].mode, st[0].nbits, st[0].rounding))
+            fn = kCompressGeneral;
+    int grid = persistent_ctas(fn);
     if (grid < 1) return LGN_ERR_CUDA;
     if ((uint32_t)grid > total_items) grid = (int)(total_items ? total_items : 1u);
-    compress_kernel<<<grid, kThreads, 0, stream>>>(
-        reinterpret_cast<WsHeader *>(base), reinterpret_cast<const LayerState *>(base + w.states),
-        reinterpret_cast<LayerDyn *>(base + w.dyn), reinterpret_cast<const Segment *>(base + w.segs),
-        L, total_items, reinterpret_cast<Partial *>(base + w.partials));
+    WsHeader *a_hdr = reinterpret_cast<WsHeader *>(base);
+    const LayerState *a_states = reinterpret_cast<const LayerState *>(base + w.states);
+    LayerDyn *a_dyn = reinterpret_cast<LayerDyn *>(base + w.dyn);
+    const Segment *a_segs = reinterpret_cast<const Segment *>(base + w.segs);
+    int a_L = L;
+    uint32_t a_items = total_items;
+    Partial *a_partials = reinterpret_cast<Partial *>(base + w.partials);
+    void *args[] = { &a_hdr, &a_states, &a_dyn, &a_segs, &a_L, &a_items, &a_partials };
+    if (cudaLaunchKernel(fn, dim3((unsigned)grid), dim3(kThreads), args, 0, stream) != cudaSuccess) return LGN_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
 }
 
@@ -549,8 +631,8 @@ extern "C" lgn_status lgn_fp_format(double mu, double sigma, int nbits, lgn_fp_f
     return LGN_OK;
 }
 
-static int apply_grid(uint32_t ntiles) {
-    int g = persistent_ctas();
+static int apply_grid(const void *fn, uint32_t ntiles) {
+    int g = persistent_ctas(fn);
     if (g < 1) return -1;
     return (uint32_t)g > ntiles ? (int)ntiles : g;
 }
@@ -566,11 +648,14 @@ extern "C" lgn_status lgn_prune(const void *g, void *out, uint64_t n, lgn_dtype 
     if (n > (1ull << 44)) return LGN_ERR_UNSUPPORTED;
     if (n == 0) return LGN_OK;
     const uint32_t ntiles = (uint32_t)((n + kTileElems - 1) / kTileElems);
-    const int grid = apply_grid(ntiles);
+    const void *fn = kPruneTable[dt];
+    const int grid = apply_grid(fn, ntiles);
     if (grid < 1) return LGN_ERR_CUDA;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (dt == LGN_BF16) prune_kernel<LGN_BF16><<<grid, kThreads, 0, st>>>(g, out, n, ntiles, snap_threshold_bf16(tau), seed);
-    else                prune_kernel<LGN_F32><<<grid, kThreads, 0, st>>>(g, out, n, ntiles, snap_threshold_f32(tau), seed);
+    float tau_used = dt == LGN_BF16 ? snap_threshold_bf16(tau) : snap_threshold_f32(tau);
+    uint32_t a_ntiles = ntiles;
+    void *args[] = { &g, &out, &n, &a_ntiles, &tau_used, &seed };
+    if (cudaLaunchKernel(fn, dim3((unsigned)grid), dim3(kThreads), args, 0, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return LGN_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
 }
 
@@ -591,13 +676,14 @@ extern "C" lgn_status lgn_quantize(const void *g, void *codes, uint64_t n, lgn_d
     if (n > (1ull << 44)) return LGN_ERR_UNSUPPORTED;
     if (n == 0) return LGN_OK;
     const uint32_t ntiles = (uint32_t)((n + kTileElems - 1) / kTileElems);
-    const int grid = apply_grid(ntiles);
+    const void *fn = kQuantizeTable[dt][2 * (fmt->nbits - 4) + (rounding == LGN_ROUND_STOCHASTIC ? 1 : 0)];
+    const int grid = apply_grid(fn, ntiles);
     if (grid < 1) return LGN_ERR_CUDA;
-    const QuantParams q = make_quant_params(*fmt);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int sr = rounding == LGN_ROUND_STOCHASTIC;
-    if (dt == LGN_BF16) quantize_kernel<LGN_BF16><<<grid, kThreads, 0, st>>>(g, codes, n, ntiles, fmt->nbits, q, sr, seed);
-    else                quantize_kernel<LGN_F32><<<grid, kThreads, 0, st>>>(g, codes, n, ntiles, fmt->nbits, q, sr, seed);
+    QuantParams q = make_quant_params(*fmt);
+    uint32_t a_ntiles = ntiles;
+    void *args[] = { &g, &codes, &n, &a_ntiles, &q, &seed };
+    if (cudaLaunchKernel(fn, dim3((unsigned)grid), dim3(kThreads), args, 0, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return LGN_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
 }
 

@@ -1,12 +1,17 @@
-// Device-side building blocks: 16-byte tile loads, the counter-based random
+// Device-side building blocks: 32-byte tile loads, the counter-based random
 // bits, and the per-tile bodies of the three O(n) passes (statistics, stochastic
-// pruning, FP quantisation + packing).  One tile = kTileElems consecutive
-// elements handled by one CTA of kThreads threads; in every load step thread t
-// of the CTA takes the t-th 16-byte vector of a kThreads*16-byte span, so each
-// warp instruction touches 512 contiguous bytes.
+// pruning, FP quantisation + packing).
+//
+// One tile = kTileElems consecutive elements handled by one CTA of kThreads
+// threads.  In every load step thread t takes the t-th 32-byte chunk of a
+// kThreads*32-byte span (one 256-bit load), so a warp instruction touches 1 KiB
+// of contiguous memory.  A chunk holds kChunk = 8 (fp32) or 16 (bf16) elements
+// and always starts at an element index that is a multiple of 8: the eight
+// elements that share one block of random bits stay in one thread.
 #pragma once
 
 #include <cstdint>
+#include <cstring>
 #include <cuda_runtime.h>
 
 #include "lgn.h"
@@ -18,93 +23,119 @@ constexpr int kWarps     = kThreads / 32;
 constexpr int kTileElems = 16384;
 
 template <int DT> struct ElemTraits;
-template <> struct ElemTraits<LGN_F32>  { static constexpr int kVec = 4; static constexpr int kBytes = 4; };
-template <> struct ElemTraits<LGN_BF16> { static constexpr int kVec = 8; static constexpr int kBytes = 2; };
+template <> struct ElemTraits<LGN_F32>  { static constexpr int kChunk = 8;  static constexpr int kBytes = 4; };
+template <> struct ElemTraits<LGN_BF16> { static constexpr int kChunk = 16; static constexpr int kBytes = 2; };
 
 __device__ __forceinline__ float    u2f(uint32_t u) { return __uint_as_float(u); }
 __device__ __forceinline__ uint32_t f2u(float f)    { return __float_as_uint(f); }
 
-// ---------------------------------------------------------------- loads / stores
-enum class Ld { Keep, Stream };   // Keep: normal L2 policy (data is read again); Stream: evict first
+struct Chunk { uint32_t w[8]; };          // 32 bytes
 
-template <Ld P>
-__device__ __forceinline__ uint4 ld16(const void *p) {
-    uint4 v;
-    if (P == Ld::Keep)
-        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    else
-        asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
-                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
+// ---------------------------------------------------------------- loads / stores
+enum class Ld { Keep, Stream };   // Keep: normal L2 policy (the tensor is read again); Stream: evict first
+
+// WIDE: one 256-bit access.  The out-of-line general tile bodies use two 128-bit
+// accesses instead (the 256-bit form is kept to code inlined into a kernel).
+template <Ld P, bool WIDE>
+__device__ __forceinline__ Chunk ld32(const void *p) {
+    Chunk c;
+    if (WIDE) {
+        if (P == Ld::Keep)
+            asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(c.w[0]), "=r"(c.w[1]), "=r"(c.w[2]), "=r"(c.w[3]),
+                           "=r"(c.w[4]), "=r"(c.w[5]), "=r"(c.w[6]), "=r"(c.w[7]) : "l"(p));
+        else
+            asm volatile("ld.global.nc.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(c.w[0]), "=r"(c.w[1]), "=r"(c.w[2]), "=r"(c.w[3]),
+                           "=r"(c.w[4]), "=r"(c.w[5]), "=r"(c.w[6]), "=r"(c.w[7]) : "l"(p));
+    } else {
+        asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(c.w[0]), "=r"(c.w[1]), "=r"(c.w[2]), "=r"(c.w[3]) : "l"(p));
+        asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4+16];"
+                     : "=r"(c.w[4]), "=r"(c.w[5]), "=r"(c.w[6]), "=r"(c.w[7]) : "l"(p));
+    }
+    return c;
 }
 
-__device__ __forceinline__ void st16_stream(void *p, const uint4 &v) {
-    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
-                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+template <bool WIDE>
+__device__ __forceinline__ void st32_stream(void *p, const Chunk &c) {
+    if (WIDE) {
+        asm volatile("st.global.L1::no_allocate.L2::evict_first.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                     :: "l"(p), "r"(c.w[0]), "r"(c.w[1]), "r"(c.w[2]), "r"(c.w[3]),
+                        "r"(c.w[4]), "r"(c.w[5]), "r"(c.w[6]), "r"(c.w[7]) : "memory");
+    } else {
+        asm volatile("st.global.cs.v4.b32 [%0], {%1,%2,%3,%4};"
+                     :: "l"(p), "r"(c.w[0]), "r"(c.w[1]), "r"(c.w[2]), "r"(c.w[3]) : "memory");
+        asm volatile("st.global.cs.v4.b32 [%0+16], {%1,%2,%3,%4};"
+                     :: "l"(p), "r"(c.w[4]), "r"(c.w[5]), "r"(c.w[6]), "r"(c.w[7]) : "memory");
+    }
 }
 
 __device__ __forceinline__ void st4_stream(void *p, uint32_t v) {
     asm volatile("st.global.cs.u32 [%0], %1;" :: "l"(p), "r"(v) : "memory");
 }
 
-// The vector of kVec elements that starts at element index `i` (a multiple of
-// kVec).  FULL: the whole vector lies inside [0, n).  Otherwise elements at or
-// past n read as zero.
+// The chunk that starts at element index i (a multiple of kChunk).  FULL: the
+// whole chunk lies inside [0, n); otherwise elements at or past n read as zero.
 template <int DT, bool FULL, Ld P>
-__device__ __forceinline__ uint4 load_vec(const void *g, uint64_t i, uint64_t n) {
-    constexpr int V = ElemTraits<DT>::kVec;
-    if (FULL || i + V <= n)
-        return ld16<P>(static_cast<const char *>(g) + i * ElemTraits<DT>::kBytes);
-    uint32_t w[4] = {0u, 0u, 0u, 0u};
+__device__ __forceinline__ Chunk load_chunk(const void *g, uint64_t i, uint64_t n) {
+    constexpr int C = ElemTraits<DT>::kChunk;
+    if (FULL || i + C <= n)
+        return ld32<P, FULL>(static_cast<const char *>(g) + i * ElemTraits<DT>::kBytes);
+    Chunk c;
+    #pragma unroll
+    for (int k = 0; k < 8; ++k) c.w[k] = 0u;
     if (DT == LGN_F32) {
         const uint32_t *p = static_cast<const uint32_t *>(g);
         #pragma unroll
-        for (int k = 0; k < 4; ++k) if (i + k < n) w[k] = p[i + k];
+        for (int k = 0; k < 8; ++k) if (i + k < n) c.w[k] = p[i + k];
     } else {
         const uint16_t *p = static_cast<const uint16_t *>(g);
         #pragma unroll
-        for (int k = 0; k < 8; ++k) if (i + k < n) w[k >> 1] |= (uint32_t)p[i + k] << ((k & 1) * 16);
+        for (int k = 0; k < 16; ++k) if (i + k < n) c.w[k >> 1] |= (uint32_t)p[i + k] << ((k & 1) * 16);
     }
-    return make_uint4(w[0], w[1], w[2], w[3]);
+    return c;
 }
 
-// Store a vector of kVec output elements of the tensor's own type at element
-// index i; elements at or past n are not written.
+// Store a chunk of output elements of the tensor's own type at element index i;
+// elements at or past n are not written.
 template <int DT, bool FULL>
-__device__ __forceinline__ void store_vec(void *out, uint64_t i, uint64_t n, const uint4 &v) {
-    constexpr int V = ElemTraits<DT>::kVec;
-    if (FULL || i + V <= n) {
-        st16_stream(static_cast<char *>(out) + i * ElemTraits<DT>::kBytes, v);
+__device__ __forceinline__ void store_chunk(void *out, uint64_t i, uint64_t n, const Chunk &c) {
+    constexpr int C = ElemTraits<DT>::kChunk;
+    if (FULL || i + C <= n) {
+        st32_stream<FULL>(static_cast<char *>(out) + i * ElemTraits<DT>::kBytes, c);
         return;
     }
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     if (DT == LGN_F32) {
         uint32_t *p = static_cast<uint32_t *>(out);
         #pragma unroll
-        for (int k = 0; k < 4; ++k) if (i + k < n) p[i + k] = w[k];
+        for (int k = 0; k < 8; ++k) if (i + k < n) p[i + k] = c.w[k];
     } else {
         uint16_t *p = static_cast<uint16_t *>(out);
         #pragma unroll
-        for (int k = 0; k < 8; ++k) if (i + k < n) p[i + k] = (uint16_t)(w[k >> 1] >> ((k & 1) * 16));
+        for (int k = 0; k < 16; ++k) if (i + k < n) p[i + k] = (uint16_t)(c.w[k >> 1] >> ((k & 1) * 16));
     }
 }
 
-// fp32 bit pattern of element k of a vector (bf16 widened exactly).
+// fp32 bit pattern of element k of a chunk (bf16 widened exactly).
 template <int DT>
-__device__ __forceinline__ uint32_t elem_bits(const uint4 &v, int k) {
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    if (DT == LGN_F32) return w[k];
-    return (k & 1) ? (w[k >> 1] & 0xFFFF0000u) : (w[k >> 1] << 16);
+__device__ __forceinline__ uint32_t elem_bits(const Chunk &c, int k) {
+    if (DT == LGN_F32) return c.w[k];
+    return (k & 1) ? (c.w[k >> 1] & 0xFFFF0000u) : (c.w[k >> 1] << 16);
 }
 
 // ---------------------------------------------------------------- random bits
-// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies
-// with the halves crossed and xored with the counter and a Weyl-stepped key.
-__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                               uint32_t k0, uint32_t k1) {
+// Philox4x32 (Salmon et al., SC'11), seven rounds: each round is two 32x32->64
+// multiplies with the halves crossed and xored with the counter and a
+// Weyl-stepped key.  One block serves eight consecutive elements, 16 bits each:
+// element 8b + e takes word e/2, low half if e is even, high half if odd.
+constexpr int kPhiloxRounds = 7;
+
+__device__ __forceinline__ uint4 rand_block(uint64_t seed, uint64_t b) {
+    uint32_t c0 = (uint32_t)b, c1 = (uint32_t)(b >> 32), c2 = 0u, c3 = 0u;
+    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
     #pragma unroll
-    for (int r = 0; r < 10; ++r) {
+    for (int r = 0; r < kPhiloxRounds; ++r) {
         unsigned long long p0 = (unsigned long long)0xD2511F53u * c0;
         unsigned long long p1 = (unsigned long long)0xCD9E8D57u * c2;
         uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
@@ -119,9 +150,24 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     return make_uint4(c0, c1, c2, c3);
 }
 
-// The four 32-bit words of elements 4b .. 4b+3 under `seed`.
-__device__ __forceinline__ uint4 rand_block(uint64_t seed, uint64_t b) {
-    return philox4x32_10((uint32_t)b, (uint32_t)(b >> 32), 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32));
+__device__ __forceinline__ uint32_t rand_word(const uint4 &r, int e) {
+    return (e >> 1) == 0 ? r.x : (e >> 1) == 1 ? r.y : (e >> 1) == 2 ? r.z : r.w;
+}
+
+// eps = h/2^16 in [0,1) for element e (0..7) of a block, built in the mantissa
+// of a float in [1,2): no integer-to-float conversion.
+__device__ __forceinline__ float eps_of(const uint4 &r, int e) {
+    const uint32_t w = rand_word(r, e);
+    const uint32_t m = (e & 1) ? ((w >> 9) & 0x007FFF80u) : ((w << 7) & 0x007FFF80u);
+    return u2f(0x3F800000u | m) - 1.0f;
+}
+
+// h * 2^(d-16): the element's 16 bits placed just below the kept mantissa bits
+// (d = dropped fraction bits of an fp32 pattern, 17..23).
+__device__ __forceinline__ uint32_t sr_addend(const uint4 &r, int e, int d) {
+    const uint32_t w = rand_word(r, e);
+    const uint32_t h = (e & 1) ? (w >> 16) : (w & 0xFFFFu);
+    return h << (d - 16);
 }
 
 // ---------------------------------------------------------------- statistics
@@ -146,26 +192,27 @@ struct StatsAcc {            // per thread, in log2 units
 //   sum y = sum d + c P,   sum y^2 = sum d^2 + 2 P sum d + c P^2.
 template <int DT, bool FULL>
 __device__ __forceinline__ void stats_tile(const void *g, uint64_t tile_base, uint64_t n, StatsAcc &acc) {
-    constexpr int V = ElemTraits<DT>::kVec;
-    constexpr int kLoads = kTileElems / (kThreads * V);   // 16 (fp32) or 8 (bf16)
-    constexpr int kGroup = 4;                             // loads in flight per thread
-    constexpr int kRunVecs = 16 / V;                      // vectors per fp32 run of 16 elements
+    constexpr int C = ElemTraits<DT>::kChunk;
+    constexpr int kLoads = kTileElems / (kThreads * C);   // 8 (fp32) or 4 (bf16)
+    constexpr int kGroup = 2;                             // 32-byte loads in flight per thread
     const float kUnset = -__int_as_float(0x7F800000);     // -inf: no nonzero seen yet
     float P = kUnset;
     double D1 = 0.0, D2 = 0.0;
-    unsigned long long C = 0;
+    unsigned long long Cn = 0;
     #pragma unroll 1
     for (int j0 = 0; j0 < kLoads; j0 += kGroup) {
-        uint4 v[kGroup];
+        Chunk v[kGroup];
         #pragma unroll
         for (int j = 0; j < kGroup; ++j)
-            v[j] = load_vec<DT, FULL, Ld::Keep>(g, tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * V, n);
+            v[j] = load_chunk<DT, FULL, Ld::Keep>(g, tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * C, n);
         #pragma unroll
-        for (int r = 0; r < kGroup / kRunVecs; ++r) {
+        for (int r = 0; r < kGroup * C / 16; ++r) {       // runs of 16 elements
             float y[16];
             #pragma unroll
-            for (int e = 0; e < 16; ++e)
-                y[e] = lg2_approx(fabsf(u2f(elem_bits<DT>(v[r * kRunVecs + e / V], e % V))));   // -inf for zero
+            for (int e = 0; e < 16; ++e) {
+                const int idx = r * 16 + e;
+                y[e] = lg2_approx(fabsf(u2f(elem_bits<DT>(v[idx / C], idx % C))));   // -inf for zero
+            }
             if (P == kUnset) {
                 #pragma unroll
                 for (int e = 0; e < 16; ++e) P = fmaxf(P, y[e]);
@@ -182,14 +229,14 @@ __device__ __forceinline__ void stats_tile(const void *g, uint64_t tile_base, ui
             }
             D1 += (double)s1;
             D2 += (double)s2;
-            C += c;
+            Cn += c;
         }
     }
-    if (C) {
-        const double p = (double)P, c = (double)C;
+    if (Cn) {
+        const double p = (double)P, c = (double)Cn;
         acc.s1 += D1 + c * p;
         acc.s2 += D2 + p * (2.0 * D1 + c * p);
-        acc.cnt += C;
+        acc.cnt += Cn;
     }
 }
 
@@ -219,60 +266,54 @@ __device__ __forceinline__ void block_reduce(StatsAcc &acc, double *sm /* 3*kWar
 }
 
 // ---------------------------------------------------------------- stochastic pruning (Eq. 5)
-__device__ __forceinline__ uint32_t prune_elem(uint32_t xb, uint32_t r, float tau, uint32_t tau_bits) {
-    float a = fabsf(u2f(xb));
-    float eps = u2f(0x3F800000u | (r >> 9)) - 1.0f;      // (r >> 9) / 2^23, exact
-    float thr = __fmul_rn(tau, eps);                     // one fp32 rounding, subnormals kept
-    uint32_t snapped = (xb & 0x80000000u) | tau_bits;
-    bool keep = a > tau;
-    bool snap = (a >= thr) && (a != 0.f);
+// keep x if |x| > alpha; else sign(x)*alpha if |x| >= fl32(alpha*eps) and x != 0; else +0.
+__device__ __forceinline__ uint32_t prune_elem(uint32_t xb, float eps, float tau, uint32_t tau_bits) {
+    const float a = fabsf(u2f(xb));
+    const float thr = __fmul_rn(tau, eps);               // one fp32 rounding, subnormals kept
+    const uint32_t snapped = (xb & 0x80000000u) | tau_bits;
+    const bool keep = a > tau;
+    const bool snap = (a >= thr) && (a != 0.f);
     return keep ? xb : (snap ? snapped : 0u);
 }
 
 template <int DT, bool FULL>
 __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t tile_base, uint64_t n,
                                            float tau, uint64_t seed) {
-    constexpr int V = ElemTraits<DT>::kVec;
-    constexpr int kLoads = kTileElems / (kThreads * V);
-    constexpr int kGroup = 4;
+    constexpr int C = ElemTraits<DT>::kChunk;
+    constexpr int kLoads = kTileElems / (kThreads * C);
+    constexpr int kGroup = 2;
     const uint32_t tau_bits = f2u(tau);
     #pragma unroll 1
     for (int j0 = 0; j0 < kLoads; j0 += kGroup) {
-        uint4 v[kGroup];
+        Chunk v[kGroup];
         #pragma unroll
         for (int j = 0; j < kGroup; ++j)
-            v[j] = load_vec<DT, FULL, Ld::Stream>(g, tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * V, n);
+            v[j] = load_chunk<DT, FULL, Ld::Stream>(g, tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * C, n);
         #pragma unroll
         for (int j = 0; j < kGroup; ++j) {
-            const uint64_t i = tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * V;
+            const uint64_t i = tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * C;
             if (!FULL && i >= n) continue;
-            uint4 o;
-            if (DT == LGN_F32) {
-                uint4 r = rand_block(seed, i >> 2);
-                o.x = prune_elem(v[j].x, r.x, tau, tau_bits);
-                o.y = prune_elem(v[j].y, r.y, tau, tau_bits);
-                o.z = prune_elem(v[j].z, r.z, tau, tau_bits);
-                o.w = prune_elem(v[j].w, r.w, tau, tau_bits);
-            } else {
-                uint4 r0 = rand_block(seed, i >> 2), r1 = rand_block(seed, (i >> 2) + 1);
-                const uint32_t rr[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
-                uint32_t w[4];
+            Chunk o;
+            #pragma unroll
+            for (int b = 0; b < C / 8; ++b) {
+                const uint4 r = rand_block(seed, (i >> 3) + b);
                 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    uint32_t lo = prune_elem(elem_bits<DT>(v[j], 2 * k), rr[2 * k], tau, tau_bits);
-                    uint32_t hi = prune_elem(elem_bits<DT>(v[j], 2 * k + 1), rr[2 * k + 1], tau, tau_bits);
-                    w[k] = (hi & 0xFFFF0000u) | (lo >> 16);
+                for (int e = 0; e < 8; ++e) {
+                    const int k = b * 8 + e;
+                    const uint32_t res = prune_elem(elem_bits<DT>(v[j], k), eps_of(r, e), tau, tau_bits);
+                    if (DT == LGN_F32) o.w[k] = res;
+                    else if ((k & 1) == 0) o.w[k >> 1] = res >> 16;
+                    else o.w[k >> 1] |= res & 0xFFFF0000u;
                 }
-                o = make_uint4(w[0], w[1], w[2], w[3]);
             }
-            store_vec<DT, FULL>(out, i, n, o);
+            store_chunk<DT, FULL>(out, i, n, o);
         }
     }
 }
 
 // ---------------------------------------------------------------- FP quantisation (Eq. 1-2, Algorithm 1)
 struct QuantParams {
-    int32_t  d;          // dropped fraction bits, 23 - man_bits
+    int32_t  d;          // dropped fraction bits of an fp32 pattern, 23 - man_bits
     int32_t  n1;         // man_bits
     int32_t  K;          // 127 + scale_exp - E_max: fp32 exponent field minus K = code exponent field
     int32_t  nfield;     // 2^exp_bits
@@ -282,13 +323,19 @@ struct QuantParams {
     uint32_t top;        // largest magnitude code
     uint32_t min_code;   // smallest normal: exponent field 1, mantissa 0
     uint32_t sign_bit;   // 1 << (nbits - 1)
+    uint32_t under_lim;  // fast path: patterns below this underflow, min(K+1, 256) << 23
+    uint32_t k_shifted;  // fast path: K << man_bits
+    float    alpha;      // smallest normal in the tensor's units, 2^(1 - E_max + scale_exp) as fp32
+    uint32_t pad[3];
 };
+static_assert(sizeof(QuantParams) == 64, "QuantParams is moved as four 16-byte words");
 
 __host__ __device__ inline QuantParams make_quant_params(const lgn_fp_format_t &f) {
     QuantParams q;
+    const int Emax = 1 << (f.exp_bits - 1);
     q.n1 = f.man_bits;
     q.d = 23 - f.man_bits;
-    q.K = 127 + f.scale_exp - (1 << (f.exp_bits - 1));
+    q.K = 127 + f.scale_exp - Emax;
     q.nfield = 1 << f.exp_bits;
     q.rtn_add = (1u << (q.d - 1)) - 1u;
     q.lsb_mask = f.man_bits > 0 ? 1u : 0u;
@@ -296,108 +343,130 @@ __host__ __device__ inline QuantParams make_quant_params(const lgn_fp_format_t &
     q.top = (((1u << f.exp_bits) - 1u) << f.man_bits) | q.man_mask;
     q.min_code = 1u << f.man_bits;
     q.sign_bit = 1u << (f.nbits - 1);
+    const int kk = q.K + 1 < 0 ? 0 : (q.K + 1 > 256 ? 256 : q.K + 1);
+    q.under_lim = (uint32_t)kk << 23;
+    q.k_shifted = q.K > 0 ? (uint32_t)q.K << f.man_bits : 0u;
+    const int ea = 1 - Emax + f.scale_exp;               // exponent of the smallest normal
+    uint32_t ab;
+    if (ea > 127) ab = 0x7F800000u;                      // beyond fp32: +inf
+    else if (ea >= -126) ab = (uint32_t)(ea + 127) << 23;
+    else if (ea >= -149) ab = 1u << (ea + 149);          // an fp32 subnormal
+    else ab = 0u;
+    memcpy(&q.alpha, &ab, 4);
+    q.pad[0] = q.pad[1] = q.pad[2] = 0u;
     return q;
 }
 
-// Code of one element from its fp32 bit pattern; integer arithmetic on the
+// Code of one element from its fp32 bit pattern, integer arithmetic on the
 // pattern: adding the rounding increment below the kept bits lets a mantissa
 // carry run into the exponent field by itself.
-template <bool SR>
-__device__ __forceinline__ uint32_t quant_elem(uint32_t xb, uint32_t r, const QuantParams &q) {
-    uint32_t mag = xb & 0x7FFFFFFFu;
-    uint32_t m = mag;
-    int K = q.K;
-    if (m < 0x00800000u) {                       // fp32 subnormal (or zero): renormalise exactly
-        m = f2u(u2f(m) * 16777216.0f);
-        K += 24;
+//
+// FAST (K >= 1, the usual case: the layer scale is not so small that fp32
+// subnormal inputs could land inside the format's range): every pattern below
+// under_lim, zero and subnormals included, underflows, so neither a zero test
+// nor renormalisation is needed, and the code is a shift and a subtraction.
+template <bool SR, bool FAST>
+__device__ __forceinline__ uint32_t quant_elem(uint32_t xb, uint32_t addend, float eps, const QuantParams &q) {
+    const uint32_t mag = xb & 0x7FFFFFFFu;
+    uint32_t code;
+    bool under;
+    if (FAST) {
+        const uint32_t add = SR ? addend : (q.rtn_add + ((mag >> q.d) & q.lsb_mask));
+        const uint32_t m2 = mag + add;
+        code = min((m2 >> q.d) - q.k_shifted, q.top);    // clip: E >= E_max, before or after the carry
+        under = mag < q.under_lim;                       // E <= -E_max before rounding
+    } else {
+        uint32_t m = mag;
+        int K = q.K;
+        if (m < 0x00800000u) {                           // fp32 subnormal (or zero): renormalise exactly
+            m = f2u(u2f(m) * 16777216.0f);
+            K += 24;
+        }
+        const uint32_t add = SR ? addend : (q.rtn_add + ((m >> q.d) & q.lsb_mask));
+        const uint32_t m2 = m + add;
+        const int f_pre = (int)(m >> 23) - K;            // E + E_max before rounding
+        const int f_post = (int)(m2 >> 23) - K;          // ... after a possible carry
+        code = ((uint32_t)f_post << q.n1) | ((m2 >> q.d) & q.man_mask);
+        if (f_post >= q.nfield) code = q.top;
+        under = (f_pre <= 0) || (mag == 0u);
     }
-    uint32_t add = SR ? (r >> (32 - q.d)) : (q.rtn_add + ((m >> q.d) & q.lsb_mask));
-    uint32_t m2 = m + add;
-    int f_pre = (int)(m >> 23) - K;              // E + E_max before rounding
-    int f_post = (int)(m2 >> 23) - K;            // ... after a possible carry
-    uint32_t code = ((uint32_t)f_post << q.n1) | ((m2 >> q.d) & q.man_mask);
-    if (f_post >= q.nfield) code = q.top;        // E >= E_max: clip
-    if (f_pre <= 0) {                            // E <= -E_max: underflow
-        if (SR) {
-            int k = 1 - f_pre;                   // smallest normal is 2^k times the binade of |x'|
-            uint32_t m24 = (m & 0x007FFFFFu) | 0x00800000u;
-            uint32_t p = m24 >> min(k - 1, 31);
-            code = ((r >> 8) < p) ? q.min_code : 0u;
+    if (under) {
+        if (SR) {                                        // Eq. 5 with alpha = the smallest normal
+            const float a = u2f(mag);
+            const float thr = __fmul_rn(q.alpha, eps);
+            code = ((a >= thr) && (mag != 0u)) ? q.min_code : 0u;
         } else {
             code = 0u;
         }
     }
-    if (mag == 0u) code = 0u;
-    if (code != 0u) code |= (xb >> 31) ? q.sign_bit : 0u;
-    return code;
+    const uint32_t sgn = (xb >> 31) ? q.sign_bit : 0u;
+    return code ? (code | sgn) : 0u;
 }
 
 // Quantise one tile and write its slice of the packed stream.  Each lane packs
-// the codes of its own vector into B = kVec*NBITS bits; 32-bit output words are
-// assembled from the lane in which they start and the one or two lanes after
-// it (warp shuffles), so every store is an aligned 32-bit word of the
-// little-endian bit stream.  `total_words` = words in the whole stream.
-template <int DT, int NBITS, bool SR, bool FULL>
+// the codes of its chunk into B = kChunk*NBITS bits (up to four 32-bit words).
+// Output words are assembled from the lane in which they start and, where B is
+// not a multiple of 32, the first bits of the next lane (one warp shuffle), so
+// every store is an aligned 32-bit word of the little-endian bit stream.
+// `total_words` = words in the whole stream.
+template <int DT, int NBITS, bool SR, bool FAST, bool FULL>
 __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint64_t tile_base, uint64_t n,
                                            uint64_t total_words, const QuantParams &q, uint64_t seed) {
-    constexpr int V = ElemTraits<DT>::kVec;
-    constexpr int B = V * NBITS;                           // bits per lane per load step
-    constexpr int kLoads = kTileElems / (kThreads * V);
-    constexpr int kGroup = 4;
+    constexpr int C = ElemTraits<DT>::kChunk;
+    constexpr int B = C * NBITS;                           // bits per lane per load step: 32..128
+    constexpr int NW = (B + 31) / 32;                      // words that hold a lane's bits
+    constexpr int kLoads = kTileElems / (kThreads * C);
+    constexpr int kGroup = 2;
     const int lane = threadIdx.x & 31;
-    const int start = lane * B;                            // lane's first bit within the warp's span
-    const int o0 = (32 - (start & 31)) & 31;               // offset of the first word that starts in this lane
-    const bool has0 = o0 < B;
-    const bool has1 = o0 + 32 < B;                         // only possible when B > 32 (bf16)
+    const int o0 = (B % 32 == 0) ? 0 : ((32 - ((lane * B) & 31)) & 31);   // first word boundary inside this lane
 
     #pragma unroll 1
     for (int j0 = 0; j0 < kLoads; j0 += kGroup) {
-        uint4 v[kGroup];
+        Chunk v[kGroup];
         #pragma unroll
         for (int j = 0; j < kGroup; ++j)
-            v[j] = load_vec<DT, FULL, Ld::Stream>(g, tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * V, n);
+            v[j] = load_chunk<DT, FULL, Ld::Stream>(g, tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * C, n);
         #pragma unroll
         for (int j = 0; j < kGroup; ++j) {
-            const uint64_t i = tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * V;
-            unsigned long long c = 0;                      // this lane's B bits
-            uint32_t rr[8];
-            if (SR) {
-                uint4 r0 = rand_block(seed, i >> 2);
-                rr[0] = r0.x; rr[1] = r0.y; rr[2] = r0.z; rr[3] = r0.w;
-                if (V == 8) {
-                    uint4 r1 = rand_block(seed, (i >> 2) + 1);
-                    rr[4] = r1.x; rr[5] = r1.y; rr[6] = r1.z; rr[7] = r1.w;
-                }
-            }
+            const uint64_t i = tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * C;
+            uint32_t cw[NW + 1];
             #pragma unroll
-            for (int k = 0; k < V; ++k) {
-                uint32_t code = quant_elem<SR>(elem_bits<DT>(v[j], k), SR ? rr[k] : 0u, q);
-                c |= (unsigned long long)code << (k * NBITS);
+            for (int k = 0; k <= NW; ++k) cw[k] = 0u;
+            #pragma unroll
+            for (int b = 0; b < C / 8; ++b) {
+                uint4 r = make_uint4(0u, 0u, 0u, 0u);
+                if (SR) r = rand_block(seed, (i >> 3) + b);
+                #pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int k = b * 8 + e;
+                    const uint32_t code = quant_elem<SR, FAST>(elem_bits<DT>(v[j], k), SR ? sr_addend(r, e, q.d) : 0u,
+                                                               SR ? eps_of(r, e) : 0.f, q);
+                    const int pos = k * NBITS;             // a constant once the loops are unrolled
+                    cw[pos >> 5] |= code << (pos & 31);
+                    if ((pos & 31) + NBITS > 32) cw[(pos >> 5) + 1] |= code >> (32 - (pos & 31));
+                }
             }
-            // first word of the warp's span, in units of 32-bit words of the stream
-            const uint64_t lane_bit = i * (uint64_t)NBITS;  // = warp span base + start
-            const uint64_t w0 = (lane_bit + o0) >> 5;
-            if constexpr (B == 32) {                        // one lane, one word
-                if (w0 < total_words) st4_stream(codes + w0, (uint32_t)c);
-            } else if constexpr (B > 32) {
-                const unsigned long long nx = __shfl_down_sync(0xFFFFFFFFu, c, 1);
-                // bits [o, o+32) of (c | nx << B)
-                if (has0) {
-                    unsigned long long win = (c >> o0) | (B - o0 < 64 ? nx << (B - o0) : 0ull);
-                    if (w0 < total_words) st4_stream(codes + w0, (uint32_t)win);
-                }
-                if (has1) {
-                    unsigned long long win = (c >> (o0 + 32)) | (nx << (B - o0 - 32));
-                    if (w0 + 1 < total_words) st4_stream(codes + w0 + 1, (uint32_t)win);
-                }
+            const uint64_t lane_bit = i * (uint64_t)NBITS;  // position of this lane's bit 0 in the stream
+            if (B % 32 == 0) {                             // whole words per lane: no neighbour needed
+                const uint64_t w0 = lane_bit >> 5;
+                #pragma unroll
+                for (int k = 0; k < NW; ++k)
+                    if (FULL || w0 + k < total_words) st4_stream(codes + w0 + k, cw[k]);
             } else {
-                const uint32_t c32 = (uint32_t)c;
-                const uint32_t n1 = __shfl_down_sync(0xFFFFFFFFu, c32, 1);
-                const uint32_t n2 = __shfl_down_sync(0xFFFFFFFFu, c32, 2);
-                if (has0) {
-                    unsigned long long win = (unsigned long long)c32 | ((unsigned long long)n1 << B)
-                                           | ((unsigned long long)n2 << (2 * B));
-                    if (w0 < total_words) st4_stream(codes + w0, (uint32_t)(win >> o0));
+                // the stream seen from this lane: its own B bits, then the next lane's
+                const uint32_t nx = __shfl_down_sync(0xFFFFFFFFu, cw[0], 1);
+                constexpr int jB = B / 32, rB = B % 32;
+                uint32_t s[NW + 1];
+                #pragma unroll
+                for (int k = 0; k <= NW; ++k)
+                    s[k] = (k < jB) ? cw[k] : (k == jB) ? (cw[jB] | (nx << rB)) : (nx >> ((32 - rB) & 31));
+                const uint64_t w0 = (lane_bit + o0) >> 5;
+                #pragma unroll
+                for (int k = 0; k < NW; ++k) {
+                    if (o0 + 32 * k < B) {
+                        const uint32_t word = __funnelshift_r(s[k], s[k + 1], o0);
+                        if (w0 + k < total_words) st4_stream(codes + w0 + k, word);
+                    }
                 }
             }
         }
