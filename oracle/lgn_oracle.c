@@ -242,17 +242,20 @@ double orc_snap_tau(double tau, int dtype)
 /* ------------------------------------------------------------------ */
 
 /* T_{alpha,eps}(x) for one element, with the element's 16 random bits h
- * given.  eps = h / 2^16 is uniform on [0,1) in steps of 2^-16.
+ * given.  eps = (h + 1) / 2^16 is uniform on (0,1] in steps of 2^-16 (never
+ * zero, so that alpha*eps > 0 and a zero can never reach the middle case).
  * The product alpha*eps is rounded once to fp32 (the precision the kernel
  * compares in); |x| and alpha are exact in fp32.
- *   |x| > alpha            -> x
- *   alpha*eps <= |x| <= alpha -> sign(x)*alpha   (x == 0 stays 0)
- *   |x| < alpha*eps        -> 0 */
+ *   alpha == 0               -> x, bit for bit (nothing is pruned)
+ *   |x| > alpha              -> x
+ *   alpha*eps <= |x| <= alpha -> sign(x)*alpha   (x == 0 stays +0)
+ *   |x| < alpha*eps          -> +0 */
 double orc_prune_one(double x, double tau_used, uint32_t h)
 {
+    if (tau_used == 0.0) return x;
     double a = fabs(x);
     if (a > tau_used) return x;
-    double eps = (double)(h & 0xFFFFu) / 65536.0;
+    double eps = (double)((h & 0xFFFFu) + 1u) / 65536.0;
     double thr = (double)(float)(tau_used * eps);   /* exact product, one rounding */
     if (a != 0.0 && a >= thr) return x < 0.0 ? -tau_used : tau_used;
     return 0.0;
@@ -363,7 +366,7 @@ enum { ORC_ROUND_NEAREST = 0, ORC_ROUND_STOCHASTIC = 1 };
  *   E <= -E_max -> 0 under round-to-nearest.  Under stochastic rounding the
  *                  value is pruned by Eq. 5 with alpha = the smallest normal
  *                  (in the tensor's own units, 2^(1-E_max+e_s) as an fp32
- *                  number) and eps = h/2^16: it becomes the smallest normal
+ *                  number) and eps = (h+1)/2^16: it becomes the smallest normal
  *                  if |x| >= fl32(alpha*eps) and 0 otherwise, exactly as
  *                  orc_prune_one decides.
  *   otherwise   -> M is rounded to n1 fraction bits (step Delta = 2^-n1).
@@ -389,7 +392,7 @@ uint32_t orc_quantize_one(double x, int n2, int n1, int e_s, int rounding, uint3
     if (E <= -Emax) {
         if (rounding != ORC_ROUND_STOCHASTIC) return 0;
         float alpha = (float)ldexp(1.0, 1 - Emax + e_s);             /* exact, or 0 / inf out of fp32 range */
-        double eps = (double)(h & 0xFFFFu) / 65536.0;
+        double eps = (double)((h & 0xFFFFu) + 1u) / 65536.0;
         double thr = (double)(float)((double)alpha * eps);
         return (fabs(x) >= thr) ? (sign | (1u << n1)) : 0u;
     }

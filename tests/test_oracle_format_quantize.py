@@ -222,7 +222,7 @@ def test_stochastic_underflow_is_eq5_with_the_smallest_normal(oracle):
             x = float(np.float32(mn * frac))
             if x == 0.0 or x >= mn:
                 continue
-            for h in [0, 1, 0x7FFF, 0x8000, 0xFFFF] + list(rs.randint(0, 65536, 40)):
+            for h in [0, 1, 0x7FFF, 0x8000, 0xFFFE, 0xFFFF] + list(rs.randint(0, 65536, 40)):
                 want = oracle.prune_one(x, float(np.float32(mn)), int(h))
                 assert want in (0.0, float(np.float32(mn)))
                 got = oracle.quantize_one(x, n2, n1, e_s, SR, int(h))
@@ -237,6 +237,7 @@ def test_stochastic_underflow_is_eq5_with_the_smallest_normal(oracle):
         hits = sum(oracle.quantize_one(x, n2, n1, e_s, SR, h) != 0 for h in range(0, 65536, 7))
         assert abs(hits / len(range(0, 65536, 7)) - x / mn) < 2e-3
     assert oracle.quantize_one(2.0 ** -7 * 2.0 ** -30, 4, 1, 0, SR, 1) == 0
+    assert oracle.quantize_one(2.0 ** -7 * 2.0 ** -16, 4, 1, 0, SR, 0) == 2       # eps = 2^-16 exactly reached
 
 
 def test_stochastic_rounding_is_unbiased(oracle):

@@ -83,7 +83,7 @@ def test_snap_tau_matches_library_roundings(oracle):
 
 
 # ------------------------------------------------------------------ Eq. 5
-H_HALF = 0x8000            # eps = 1/2 (16 random bits per element)
+H_HALF = 0x7FFF            # eps = (h + 1) / 2^16 = 1/2
 
 
 def test_prune_hand_cases(oracle):
@@ -93,22 +93,24 @@ def test_prune_hand_cases(oracle):
         (-0.5, 1.0, H_HALF, -1.0),          # |x| == alpha*eps is kept
         (1.0, 1.0, H_HALF, 1.0),            # |x| == alpha maps to alpha
         (-1.5, 1.0, H_HALF, -1.5),
-        (0.0, 1.0, 0, 0.0),                 # eps = 0: zero still stays zero
-        (1e-30, 1.0, 0, 1.0),               # eps = 0: every nonzero |x| <= alpha snaps
-        (1e-30, 1.0, 1, 0.0),               # eps = 2^-16
-        (0.9999, 1.0, 0xFFFF, 0.0),         # eps = 1 - 2^-16 > 0.9999
+        (0.0, 1.0, 0, 0.0),                 # zero stays zero whatever eps
+        (2.0 ** -16, 1.0, 0, 1.0),          # eps = 2^-16, the smallest
+        (2.0 ** -17, 1.0, 0, 0.0),
+        (0.99999, 1.0, 0xFFFF, 0.0),        # eps = 1: only |x| == alpha survives
+        (1.0, 1.0, 0xFFFF, 1.0),
         (3.0, 0.0, H_HALF, 3.0),            # tau = 0: identity
         (0.0, 0.0, H_HALF, 0.0),
     ]
     for x, tau, h, want in cases:
         assert oracle.prune_one(float(np.float32(x)), tau, h) == float(np.float32(want))
-    assert math.copysign(1.0, oracle.prune_one(-0.0, 1.0, 0)) == 1.0     # -0 -> +0
+    assert math.copysign(1.0, oracle.prune_one(-0.0, 1.0, 0)) == 1.0      # -0 -> +0 when pruning
+    assert math.copysign(1.0, oracle.prune_one(-0.0, 0.0, 0)) == -1.0     # tau = 0 changes nothing at all
 
 
 def test_prune_threshold_product_is_rounded_to_fp32(oracle):
     tau = float(np.float32(1.0 + 2 ** -23))
-    h = 0x5555
-    eps = h / 2 ** 16
+    h = 0x5554
+    eps = (h + 1) / 2 ** 16
     thr32 = float(np.float32(tau) * np.float32(eps))            # numpy's fp32 multiply
     exact = tau * eps
     assert thr32 != exact
@@ -174,5 +176,6 @@ def test_prune_achieves_requested_sparsity(oracle, mu, sigma, l, S):
 
 def test_prune_tau_zero_is_identity(oracle):
     g = synth.as_numpy_bits(synth.lognormal_tensor(10_000, -12.0, 2.0, 0.5, seed=8))
+    g[:3] = [-0.0, 0.0, -1e-30]
     out = oracle.prune(g, 0.0, seed=1)
-    assert np.array_equal(out, g)
+    assert np.array_equal(out.view(np.uint32), g.view(np.uint32))
