@@ -30,7 +30,8 @@ namespace lgn {
 struct WsHeader {
     uint32_t queue_head;
     uint32_t error;
-    uint32_t pad[62];
+    Weyl     weyl;                       // key-schedule increments, read as run-time values
+    uint32_t pad[60];
 };
 static_assert(sizeof(WsHeader) == 256, "header is one 256-byte block");
 
@@ -131,67 +132,88 @@ __device__ __forceinline__ void st_release(uint32_t *p, uint32_t v) {
 
 // ------------------------------------------------------------------ tile runners
 // Every pass has one hot body (whole tile inside the tensor; for quantisation
-// also the fast code path) that specialised kernels inline, and one general body
-// (ragged last tile, any layer scale) kept out of line so that it costs the hot
-// path no registers.
+// also the fast code path, for pruning a normal-range threshold) that
+// specialised kernels inline, and one general body (ragged last tile, any layer
+// scale, any threshold) kept out of line so that it costs the hot path no
+// registers.
 template <int DT>
 __device__ __noinline__ void stats_tile_general(const void *g, uint64_t base, uint64_t n, StatsAcc &acc) {
     stats_tile<DT, false>(g, base, n, acc);
 }
 
+// One tile's sums: per-warp shuffle tree, eight warp results through shared
+// memory, added in warp order by thread 0, which also stores the tile's partial.
+// One barrier; `sm` is reused only after the caller's next barrier.
 template <int DT, bool INLINE_HOT>
 __device__ __forceinline__ void run_stats_tile(const LayerState &L, uint32_t tile, Partial *partials, double *sm) {
     StatsAcc acc;
     const uint64_t base = (uint64_t)tile * kTileElems;
     if (INLINE_HOT && base + kTileElems <= L.n) stats_tile<DT, true>(L.g, base, L.n, acc);
     else                                        stats_tile_general<DT>(L.g, base, L.n, acc);
-    block_reduce(acc, sm);
+    #pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        acc.s1 += __shfl_down_sync(0xFFFFFFFFu, acc.s1, off);
+        acc.s2 += __shfl_down_sync(0xFFFFFFFFu, acc.s2, off);
+        acc.cnt += __shfl_down_sync(0xFFFFFFFFu, acc.cnt, off);
+    }
+    const int w = threadIdx.x >> 5;
+    if ((threadIdx.x & 31) == 0) {
+        sm[w] = acc.s1; sm[kWarps + w] = acc.s2; sm[2 * kWarps + w] = __longlong_as_double((long long)acc.cnt);
+    }
+    __syncthreads();
     if (threadIdx.x == 0) {
         Partial p;
-        p.s1 = acc.s1; p.s2 = acc.s2; p.cnt = acc.cnt; p.pad = 0;
+        p.s1 = 0.0; p.s2 = 0.0; p.cnt = 0; p.pad = 0;
+        #pragma unroll
+        for (int k = 0; k < kWarps; ++k) {
+            p.s1 += sm[k]; p.s2 += sm[kWarps + k];
+            p.cnt += (unsigned long long)__double_as_longlong(sm[2 * kWarps + k]);
+        }
         partials[L.partial0 + tile] = p;
     }
 }
 
 template <int DT>
 __device__ __noinline__ void prune_tile_general(const void *g, void *out, uint64_t base, uint64_t n,
-                                                float tau, uint64_t seed) {
-    prune_tile<DT, false>(g, out, base, n, tau, seed);
+                                                float tau, uint64_t seed, const Weyl &wy) {
+    prune_tile<DT, false>(g, out, base, n, tau, seed, wy);
 }
 
 template <int DT, bool INLINE_HOT>
 __device__ __forceinline__ void run_prune_tile(const void *g, void *out, uint64_t n, uint32_t tile,
-                                               float tau, uint64_t seed) {
+                                               float tau, uint64_t seed, const Weyl &wy) {
     const uint64_t base = (uint64_t)tile * kTileElems;
-    if (INLINE_HOT && base + kTileElems <= n) prune_tile<DT, true>(g, out, base, n, tau, seed);
-    else                                      prune_tile_general<DT>(g, out, base, n, tau, seed);
+    const bool tiny = tau > 0.f && tau < 1.17549435e-38f;     // alpha*eps could round to zero
+    if (INLINE_HOT && base + kTileElems <= n && !tiny) prune_tile<DT, true>(g, out, base, n, tau, seed, wy);
+    else                                               prune_tile_general<DT>(g, out, base, n, tau, seed, wy);
 }
 
 template <int DT, int NBITS, bool SR>
 __device__ __noinline__ void quant_tile_general(const void *g, uint32_t *codes, uint64_t base, uint64_t n,
-                                                uint64_t total_words, const QuantParams &q, uint64_t seed) {
-    quant_tile<DT, NBITS, SR, false, false>(g, codes, base, n, total_words, q, seed);
+                                                uint64_t total_words, const QuantParams &q, uint64_t seed,
+                                                const Weyl &wy) {
+    quant_tile<DT, NBITS, SR, false, false>(g, codes, base, n, total_words, q, seed, wy);
 }
 
 template <int DT, int NBITS, bool SR, bool INLINE_HOT>
 __device__ __forceinline__ void run_quant_tile(const void *g, void *out, uint64_t n, uint32_t tile,
-                                               const QuantParams &q, uint64_t seed) {
+                                               const QuantParams &q, uint64_t seed, const Weyl &wy) {
     const uint64_t base = (uint64_t)tile * kTileElems;
     const uint64_t total_words = (n * (uint64_t)NBITS + 31) >> 5;
     uint32_t *codes = static_cast<uint32_t *>(out);
     if (INLINE_HOT && base + kTileElems <= n && q.K >= 1)
-        quant_tile<DT, NBITS, SR, true, true>(g, codes, base, n, total_words, q, seed);
+        quant_tile<DT, NBITS, SR, true, true>(g, codes, base, n, total_words, q, seed, wy);
     else
-        quant_tile_general<DT, NBITS, SR>(g, codes, base, n, total_words, q, seed);
+        quant_tile_general<DT, NBITS, SR>(g, codes, base, n, total_words, q, seed, wy);
 }
 
 // run-time dispatch for groups whose layers differ in type, mode or width
 template <int DT>
 __device__ __forceinline__ void run_quant_tile_any(const void *g, void *out, uint64_t n, uint32_t tile, int nbits,
-                                                   const QuantParams &q, bool sr, uint64_t seed) {
+                                                   const QuantParams &q, bool sr, uint64_t seed, const Weyl &wy) {
     #define LGN_Q(NB) \
-        if (sr) run_quant_tile<DT, NB, true, false>(g, out, n, tile, q, seed); \
-        else    run_quant_tile<DT, NB, false, false>(g, out, n, tile, q, seed);
+        if (sr) run_quant_tile<DT, NB, true, false>(g, out, n, tile, q, seed, wy); \
+        else    run_quant_tile<DT, NB, false, false>(g, out, n, tile, q, seed, wy);
     switch (nbits) {
         case 4: LGN_Q(4) break;
         case 5: LGN_Q(5) break;
@@ -281,6 +303,7 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
                 int num_layers, uint32_t total_items, Partial *partials) {
     __shared__ double sm_red[3 * kWarps];
     __shared__ uint32_t sm_item[2];
+    __shared__ uint32_t sm_fin[2];               // layer + 1 whose statistics this CTA has just completed
     __shared__ uint32_t sm_flag;
     constexpr bool kSpecial = DT != kAny;
 
@@ -300,12 +323,26 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
             }
         }
     }
+    Weyl wy;
+    wy.w0 = __ldcg(&hdr->weyl.w0);
+    wy.w1 = __ldcg(&hdr->weyl.w1);
 
+    // Thread 0 keeps one queue item in hand: the next pop is issued as soon as
+    // the current item is known, so its latency hides behind the tile's work.
+    uint32_t next_item = 0, fin_layer1 = 0;      // thread 0 only
+    if (threadIdx.x == 0) next_item = atomicAdd(&hdr->queue_head, 1u);
     uint32_t seg = 0;
+    int ready_layer = -1;                        // layer whose closed form this CTA has already seen published
     for (uint32_t it = 0;; ++it) {
-        if (threadIdx.x == 0) sm_item[it & 1] = atomicAdd(&hdr->queue_head, 1u);
+        if (threadIdx.x == 0) { sm_item[it & 1] = next_item; sm_fin[it & 1] = fin_layer1; fin_layer1 = 0; }
         __syncthreads();
         const uint32_t item = sm_item[it & 1];
+        const uint32_t fin = sm_fin[it & 1];
+        if (threadIdx.x == 0 && item < total_items) next_item = atomicAdd(&hdr->queue_head, 1u);
+        if (fin) {                               // this CTA stored the last partial of layer fin-1
+            __threadfence();
+            finalize_layer(states[fin - 1], dyn + (fin - 1), partials, sm_red);
+        }
         if (item >= total_items) break;
         while (item >= segs[seg].first_item + segs[seg].ntiles) ++seg;
         const Segment sg = segs[seg];
@@ -325,44 +362,41 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
             if (threadIdx.x == 0) {
                 __threadfence();                                   // the partial before the ticket
                 const uint32_t ticket = atomicAdd(&D->done, 1u);
-                sm_flag = (ticket == L.ntiles - 1u);
-            }
-            __syncthreads();
-            if (sm_flag) {
-                __threadfence();
-                finalize_layer(L, D, partials, sm_red);
+                if (ticket == L.ntiles - 1u) fin_layer1 = sg.layer + 1u;   // acted on at the next barrier
             }
         } else {
-            if (threadIdx.x == 0) {
-                uint32_t polls = 0, ok = 1;
-                while (ld_acquire(&D->ready) == 0u) {
-                    if (++polls > kMaxPolls || *(volatile uint32_t *)&hdr->error) { ok = 0; break; }
-                    __nanosleep(200);
-                }
-                if (!ok) {
-                    atomicExch(&hdr->error, 1u);
-                    if (L.result_out) *(volatile int32_t *)&L.result_out->status = LGN_ERR_TIMEOUT;
-                }
-                sm_flag = ok;
-            }
-            __syncthreads();
-            if (sm_flag) {
-                if constexpr (kSpecial && MODE == LGN_MODE_PRUNE) {
-                    run_prune_tile<DT, true>(L.g, L.out, L.n, tile, __ldcg(&D->tau), L.seed);
-                } else if constexpr (kSpecial && MODE == LGN_MODE_QUANTIZE) {
-                    const QuantParams q = load_quant_params(D);
-                    run_quant_tile<DT, NBITS, SR != 0, true>(L.g, L.out, L.n, tile, q, L.seed);
-                } else if constexpr (!kSpecial) {
-                    if (L.mode == LGN_MODE_PRUNE) {
-                        const float tau = __ldcg(&D->tau);
-                        if (L.dt == LGN_BF16) run_prune_tile<LGN_BF16, false>(L.g, L.out, L.n, tile, tau, L.seed);
-                        else                  run_prune_tile<LGN_F32, false>(L.g, L.out, L.n, tile, tau, L.seed);
-                    } else {
-                        const QuantParams q = load_quant_params(D);
-                        const bool sr = L.rounding == LGN_ROUND_STOCHASTIC;
-                        if (L.dt == LGN_BF16) run_quant_tile_any<LGN_BF16>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed);
-                        else                  run_quant_tile_any<LGN_F32>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed);
+            if ((int)sg.layer != ready_layer) {
+                if (threadIdx.x == 0) {
+                    uint32_t polls = 0, ok = 1;
+                    while (ld_acquire(&D->ready) == 0u) {
+                        if (++polls > kMaxPolls || *(volatile uint32_t *)&hdr->error) { ok = 0; break; }
+                        __nanosleep(100);
                     }
+                    if (!ok) {
+                        atomicExch(&hdr->error, 1u);
+                        if (L.result_out) *(volatile int32_t *)&L.result_out->status = LGN_ERR_TIMEOUT;
+                    }
+                    sm_flag = ok;
+                }
+                __syncthreads();
+                if (!sm_flag) continue;                            // timed out: skip the tile, keep draining
+                ready_layer = (int)sg.layer;
+            }
+            if constexpr (kSpecial && MODE == LGN_MODE_PRUNE) {
+                run_prune_tile<DT, true>(L.g, L.out, L.n, tile, __ldcg(&D->tau), L.seed, wy);
+            } else if constexpr (kSpecial && MODE == LGN_MODE_QUANTIZE) {
+                const QuantParams q = load_quant_params(D);
+                run_quant_tile<DT, NBITS, SR != 0, true>(L.g, L.out, L.n, tile, q, L.seed, wy);
+            } else if constexpr (!kSpecial) {
+                if (L.mode == LGN_MODE_PRUNE) {
+                    const float tau = __ldcg(&D->tau);
+                    if (L.dt == LGN_BF16) run_prune_tile<LGN_BF16, false>(L.g, L.out, L.n, tile, tau, L.seed, wy);
+                    else                  run_prune_tile<LGN_F32, false>(L.g, L.out, L.n, tile, tau, L.seed, wy);
+                } else {
+                    const QuantParams q = load_quant_params(D);
+                    const bool sr = L.rounding == LGN_ROUND_STOCHASTIC;
+                    if (L.dt == LGN_BF16) run_quant_tile_any<LGN_BF16>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed, wy);
+                    else                  run_quant_tile_any<LGN_F32>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed, wy);
                 }
             }
         }
@@ -372,17 +406,17 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
 // ------------------------------------------------------------------ stand-alone apply kernels
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 4)
-prune_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, float tau, uint64_t seed) {
+prune_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, float tau, uint64_t seed, Weyl wy) {
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)
-        run_prune_tile<DT, true>(g, out, n, tile, tau, seed);
+        run_prune_tile<DT, true>(g, out, n, tile, tau, seed, wy);
 }
 
 template <int DT, int NBITS, int SR>
 __global__ void __launch_bounds__(kThreads, 4)
 quantize_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, const __grid_constant__ QuantParams q,
-                uint64_t seed) {
+                uint64_t seed, Weyl wy) {
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)
-        run_quant_tile<DT, NBITS, SR != 0, true>(g, out, n, tile, q, seed);
+        run_quant_tile<DT, NBITS, SR != 0, true>(g, out, n, tile, q, seed, wy);
 }
 
 // ------------------------------------------------------------------ kernel tables
@@ -526,6 +560,12 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
 
     // image of [header | states | dyn (zero) | segments]
     std::vector<unsigned char> image(w.partials, 0);
+    {
+        WsHeader h;
+        memset(&h, 0, sizeof h);
+        h.weyl.w0 = kWeyl0; h.weyl.w1 = kWeyl1;
+        memcpy(image.data(), &h, sizeof h);
+    }
     memcpy(image.data() + w.states, st.data(), sizeof(LayerState) * (size_t)L);
     memcpy(image.data() + w.segs, segs.data(), sizeof(Segment) * segs.size());
     const size_t used = upload_bytes(w, L);
@@ -653,7 +693,8 @@ extern "C" lgn_status lgn_prune(const void *g, void *out, uint64_t n, lgn_dtype 
     if (grid < 1) return LGN_ERR_CUDA;
     float tau_used = dt == LGN_BF16 ? snap_threshold_bf16(tau) : snap_threshold_f32(tau);
     uint32_t a_ntiles = ntiles;
-    void *args[] = { &g, &out, &n, &a_ntiles, &tau_used, &seed };
+    Weyl wy = { kWeyl0, kWeyl1 };
+    void *args[] = { &g, &out, &n, &a_ntiles, &tau_used, &seed, &wy };
     if (cudaLaunchKernel(fn, dim3((unsigned)grid), dim3(kThreads), args, 0, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return LGN_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
@@ -681,7 +722,8 @@ extern "C" lgn_status lgn_quantize(const void *g, void *codes, uint64_t n, lgn_d
     if (grid < 1) return LGN_ERR_CUDA;
     QuantParams q = make_quant_params(*fmt);
     uint32_t a_ntiles = ntiles;
-    void *args[] = { &g, &codes, &n, &a_ntiles, &q, &seed };
+    Weyl wy = { kWeyl0, kWeyl1 };
+    void *args[] = { &g, &codes, &n, &a_ntiles, &q, &seed, &wy };
     if (cudaLaunchKernel(fn, dim3((unsigned)grid), dim3(kThreads), args, 0, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return LGN_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;

@@ -131,21 +131,26 @@ __device__ __forceinline__ uint32_t elem_bits(const Chunk &c, int k) {
 // element 8b + e takes word e/2, low half if e is even, high half if odd.
 constexpr int kPhiloxRounds = 7;
 
-__device__ __forceinline__ uint4 rand_block(uint64_t seed, uint64_t b) {
+// The two Weyl increments of the key schedule.  They are handed to the kernels
+// as run-time values (not literals) so that round r's key is formed as
+// key + r*W by the multiply-add pipe instead of by a chain of integer adds on
+// the busier ALU pipe.
+struct Weyl { uint32_t w0, w1; };
+constexpr uint32_t kWeyl0 = 0x9E3779B9u, kWeyl1 = 0xBB67AE85u;
+
+__device__ __forceinline__ uint4 rand_block(uint64_t seed, uint64_t b, const Weyl &wy) {
     uint32_t c0 = (uint32_t)b, c1 = (uint32_t)(b >> 32), c2 = 0u, c3 = 0u;
-    uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+    const uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
     #pragma unroll
     for (int r = 0; r < kPhiloxRounds; ++r) {
-        unsigned long long p0 = (unsigned long long)0xD2511F53u * c0;
-        unsigned long long p1 = (unsigned long long)0xCD9E8D57u * c2;
-        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
-        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        const unsigned long long p0 = (unsigned long long)0xD2511F53u * c0;
+        const unsigned long long p1 = (unsigned long long)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ (k0 + (uint32_t)r * wy.w0);
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ (k1 + (uint32_t)r * wy.w1);
         c1 = (uint32_t)p1;
         c3 = (uint32_t)p0;
         c0 = n0;
         c2 = n2;
-        k0 += 0x9E3779B9u;
-        k1 += 0xBB67AE85u;
     }
     return make_uint4(c0, c1, c2, c3);
 }
@@ -154,20 +159,20 @@ __device__ __forceinline__ uint32_t rand_word(const uint4 &r, int e) {
     return (e >> 1) == 0 ? r.x : (e >> 1) == 1 ? r.y : (e >> 1) == 2 ? r.z : r.w;
 }
 
-// eps = h/2^16 in [0,1) for element e (0..7) of a block, built in the mantissa
-// of a float in [1,2): no integer-to-float conversion.
-__device__ __forceinline__ float eps_of(const uint4 &r, int e) {
+// The element's 16 random bits as an integer and as a float (the conversion of a
+// 16-bit half of a register is one instruction on the otherwise idle
+// conversion unit).
+__device__ __forceinline__ uint32_t rand_h(const uint4 &r, int e) {
     const uint32_t w = rand_word(r, e);
-    const uint32_t m = (e & 1) ? ((w >> 9) & 0x007FFF80u) : ((w << 7) & 0x007FFF80u);
-    return u2f(0x3F800000u | m) - 1.0f;
+    return (e & 1) ? (w >> 16) : (w & 0xFFFFu);
 }
-
-// h * 2^(d-16): the element's 16 bits placed just below the kept mantissa bits
-// (d = dropped fraction bits of an fp32 pattern, 17..23).
-__device__ __forceinline__ uint32_t sr_addend(const uint4 &r, int e, int d) {
+__device__ __forceinline__ float rand_hf(const uint4 &r, int e) {
     const uint32_t w = rand_word(r, e);
-    const uint32_t h = (e & 1) ? (w >> 16) : (w & 0xFFFFu);
-    return h << (d - 16);
+    return (e & 1) ? (float)(unsigned short)(w >> 16) : (float)(unsigned short)(w & 0xFFFFu);
+}
+// eps = (h + 1) / 2^16 in (0,1]: exact in fp32.
+__device__ __forceinline__ float eps_of(const uint4 &r, int e) {
+    return fmaf(rand_hf(r, e), 0x1p-16f, 0x1p-16f);
 }
 
 // ---------------------------------------------------------------- statistics
@@ -217,16 +222,17 @@ __device__ __forceinline__ void stats_tile(const void *g, uint64_t tile_base, ui
                 #pragma unroll
                 for (int e = 0; e < 16; ++e) P = fmaxf(P, y[e]);
             }
-            float s1 = 0.f, s2 = 0.f;
-            uint32_t c = 0;
+            float s1 = 0.f, s2 = 0.f, cf = 0.f;            // cf: nonzeros of this run, exact in fp32
             #pragma unroll
             for (int e = 0; e < 16; ++e) {
-                bool nz = y[e] != kUnset;
-                float d = nz ? y[e] - P : 0.f;
-                s1 += d;
-                s2 = fmaf(d, d, s2);
-                c += nz ? 1u : 0u;
+                if (y[e] != kUnset) {                      // predicated: no select, no integer add
+                    const float d = y[e] - P;
+                    s1 += d;
+                    s2 = fmaf(d, d, s2);
+                    cf += 1.0f;
+                }
             }
+            const uint32_t c = (uint32_t)cf;
             D1 += (double)s1;
             D2 += (double)s2;
             Cn += c;
@@ -266,23 +272,29 @@ __device__ __forceinline__ void block_reduce(StatsAcc &acc, double *sm /* 3*kWar
 }
 
 // ---------------------------------------------------------------- stochastic pruning (Eq. 5)
-// keep x if |x| > alpha; else sign(x)*alpha if |x| >= fl32(alpha*eps) and x != 0; else +0.
-__device__ __forceinline__ uint32_t prune_elem(uint32_t xb, float eps, float tau, uint32_t tau_bits) {
+// With a = |x| and thr = fl32(alpha*eps) <= alpha, Eq. 5 is
+//     out = (a >= thr) ? sign(x) * max(a, alpha) : +0
+// (a > alpha passes both tests and max keeps a; thr <= a <= alpha gives alpha).
+// ZCHECK adds the explicit "a zero stays zero" test that is needed only when
+// alpha is so small that alpha*eps can round to zero.
+template <bool ZCHECK>
+__device__ __forceinline__ uint32_t prune_elem(uint32_t xb, float eps, float tau) {
     const float a = fabsf(u2f(xb));
     const float thr = __fmul_rn(tau, eps);               // one fp32 rounding, subnormals kept
-    const uint32_t snapped = (xb & 0x80000000u) | tau_bits;
-    const bool keep = a > tau;
-    const bool snap = (a >= thr) && (a != 0.f);
-    return keep ? xb : (snap ? snapped : 0u);
+    bool p = a >= thr;
+    if (ZCHECK) p = p && (a != 0.f);
+    const uint32_t kept = (xb & 0x80000000u) | f2u(fmaxf(a, tau));
+    return p ? kept : 0u;
 }
 
+// tau == 0 never reaches this function (the caller copies the tile instead).
 template <int DT, bool FULL>
 __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t tile_base, uint64_t n,
-                                           float tau, uint64_t seed) {
+                                           float tau, uint64_t seed, const Weyl &wy) {
     constexpr int C = ElemTraits<DT>::kChunk;
     constexpr int kLoads = kTileElems / (kThreads * C);
     constexpr int kGroup = 2;
-    const uint32_t tau_bits = f2u(tau);
+    constexpr bool ZCHECK = !FULL;                        // the general body also serves tiny thresholds
     #pragma unroll 1
     for (int j0 = 0; j0 < kLoads; j0 += kGroup) {
         Chunk v[kGroup];
@@ -294,16 +306,20 @@ __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t ti
             const uint64_t i = tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * C;
             if (!FULL && i >= n) continue;
             Chunk o;
-            #pragma unroll
-            for (int b = 0; b < C / 8; ++b) {
-                const uint4 r = rand_block(seed, (i >> 3) + b);
+            if (tau == 0.f) {
+                o = v[j];                                  // alpha = 0: the tensor is left as it is
+            } else {
                 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int k = b * 8 + e;
-                    const uint32_t res = prune_elem(elem_bits<DT>(v[j], k), eps_of(r, e), tau, tau_bits);
-                    if (DT == LGN_F32) o.w[k] = res;
-                    else if ((k & 1) == 0) o.w[k >> 1] = res >> 16;
-                    else o.w[k >> 1] |= res & 0xFFFF0000u;
+                for (int b = 0; b < C / 8; ++b) {
+                    const uint4 r = rand_block(seed, (i >> 3) + b, wy);
+                    #pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const int k = b * 8 + e;
+                        const uint32_t res = prune_elem<ZCHECK>(elem_bits<DT>(v[j], k), eps_of(r, e), tau);
+                        if (DT == LGN_F32) o.w[k] = res;
+                        else if ((k & 1) == 0) o.w[k >> 1] = res >> 16;
+                        else o.w[k >> 1] |= res & 0xFFFF0000u;
+                    }
                 }
             }
             store_chunk<DT, FULL>(out, i, n, o);
@@ -323,10 +339,11 @@ struct QuantParams {
     uint32_t top;        // largest magnitude code
     uint32_t min_code;   // smallest normal: exponent field 1, mantissa 0
     uint32_t sign_bit;   // 1 << (nbits - 1)
-    uint32_t under_lim;  // fast path: patterns below this underflow, min(K+1, 256) << 23
-    uint32_t k_shifted;  // fast path: K << man_bits
+    int32_t  k23;        // fast path: min(K, 255) << 23, taken off the pattern before the shift
+    uint32_t sr_mult;    // fast path: 2^(d-16), places the 16 random bits below the kept bits
     float    alpha;      // smallest normal in the tensor's units, 2^(1 - E_max + scale_exp) as fp32
-    uint32_t pad[3];
+    uint32_t one;        // the value 1, as a run-time operand (see quant_elem)
+    uint32_t pad[2];
 };
 static_assert(sizeof(QuantParams) == 64, "QuantParams is moved as four 16-byte words");
 
@@ -343,9 +360,8 @@ __host__ __device__ inline QuantParams make_quant_params(const lgn_fp_format_t &
     q.top = (((1u << f.exp_bits) - 1u) << f.man_bits) | q.man_mask;
     q.min_code = 1u << f.man_bits;
     q.sign_bit = 1u << (f.nbits - 1);
-    const int kk = q.K + 1 < 0 ? 0 : (q.K + 1 > 256 ? 256 : q.K + 1);
-    q.under_lim = (uint32_t)kk << 23;
-    q.k_shifted = q.K > 0 ? (uint32_t)q.K << f.man_bits : 0u;
+    q.k23 = (q.K < 0 ? 0 : (q.K > 255 ? 255 : q.K)) << 23;
+    q.sr_mult = 1u << (q.d - 16);
     const int ea = 1 - Emax + f.scale_exp;               // exponent of the smallest normal
     uint32_t ab;
     if (ea > 127) ab = 0x7F800000u;                      // beyond fp32: +inf
@@ -353,54 +369,65 @@ __host__ __device__ inline QuantParams make_quant_params(const lgn_fp_format_t &
     else if (ea >= -149) ab = 1u << (ea + 149);          // an fp32 subnormal
     else ab = 0u;
     memcpy(&q.alpha, &ab, 4);
-    q.pad[0] = q.pad[1] = q.pad[2] = 0u;
+    q.one = 1u;
+    q.pad[0] = q.pad[1] = 0u;
     return q;
 }
 
 // Code of one element from its fp32 bit pattern, integer arithmetic on the
 // pattern: adding the rounding increment below the kept bits lets a mantissa
-// carry run into the exponent field by itself.
+// carry run into the exponent field by itself.  h = the element's 16 random
+// bits, eps = (h+1)/2^16 (both unused for round-to-nearest).
 //
 // FAST (K >= 1, the usual case: the layer scale is not so small that fp32
-// subnormal inputs could land inside the format's range): every pattern below
-// under_lim, zero and subnormals included, underflows, so neither a zero test
-// nor renormalisation is needed, and the code is a shift and a subtraction.
+// subnormal inputs could land inside the format's range).  With the pattern
+// taken as a signed integer and K << 23 subtracted, the arithmetic shift by d
+// gives [E + E_max | mantissa] directly; it is <= min_code exactly for the
+// values that underflow (E <= -E_max) and > top exactly for those that clip, so
+// one clamp to [min_code, top] settles both, and a value that underflows is
+// then either zeroed or left at min_code (stochastic survival, Eq. 5 with
+// alpha = the smallest normal).  The additions are written as multiply-adds
+// with the run-time operand q.one so that they issue on the multiply-add pipe
+// and leave the integer ALU, the bottleneck of this kernel, to the shifts,
+// clamps and selects.
 template <bool SR, bool FAST>
-__device__ __forceinline__ uint32_t quant_elem(uint32_t xb, uint32_t addend, float eps, const QuantParams &q) {
+__device__ __forceinline__ uint32_t quant_elem(uint32_t xb, uint32_t h, float eps, const QuantParams &q) {
     const uint32_t mag = xb & 0x7FFFFFFFu;
-    uint32_t code;
-    bool under;
+    const float a = u2f(mag);
     if (FAST) {
-        const uint32_t add = SR ? addend : (q.rtn_add + ((mag >> q.d) & q.lsb_mask));
-        const uint32_t m2 = mag + add;
-        code = min((m2 >> q.d) - q.k_shifted, q.top);    // clip: E >= E_max, before or after the carry
-        under = mag < q.under_lim;                       // E <= -E_max before rounding
-    } else {
-        uint32_t m = mag;
-        int K = q.K;
-        if (m < 0x00800000u) {                           // fp32 subnormal (or zero): renormalise exactly
-            m = f2u(u2f(m) * 16777216.0f);
-            K += 24;
-        }
-        const uint32_t add = SR ? addend : (q.rtn_add + ((m >> q.d) & q.lsb_mask));
-        const uint32_t m2 = m + add;
-        const int f_pre = (int)(m >> 23) - K;            // E + E_max before rounding
-        const int f_post = (int)(m2 >> 23) - K;          // ... after a possible carry
-        code = ((uint32_t)f_post << q.n1) | ((m2 >> q.d) & q.man_mask);
-        if (f_post >= q.nfield) code = q.top;
-        under = (f_pre <= 0) || (mag == 0u);
-    }
-    if (under) {
-        if (SR) {                                        // Eq. 5 with alpha = the smallest normal
-            const float a = u2f(mag);
-            const float thr = __fmul_rn(q.alpha, eps);
-            code = ((a >= thr) && (mag != 0u)) ? q.min_code : 0u;
+        int m2;
+        if (SR) {
+            const int base = (int)(mag * q.one) - q.k23;
+            m2 = (int)(h * q.sr_mult) + base;
         } else {
-            code = 0u;
+            const uint32_t lsb = (mag >> q.d) & q.lsb_mask;
+            const int base = (int)(mag * q.one) + (int)q.rtn_add - q.k23;
+            m2 = (int)(lsb * q.one) + base;
         }
+        const int raw = m2 >> q.d;                                        // arithmetic shift
+        const uint32_t code = (uint32_t)min(max(raw, (int)q.min_code), (int)q.top);
+        bool kill = a < q.alpha;                                          // E <= -E_max: underflow
+        if (SR) kill = kill && (a < __fmul_rn(q.alpha, eps));             // ... unless it survives
+        const uint32_t comb = (xb >> 31) * q.sign_bit + code;
+        return kill ? 0u : comb;
     }
-    const uint32_t sgn = (xb >> 31) ? q.sign_bit : 0u;
-    return code ? (code | sgn) : 0u;
+    uint32_t m = mag;
+    int K = q.K;
+    if (m < 0x00800000u) {                               // fp32 subnormal (or zero): renormalise exactly
+        m = f2u(u2f(m) * 16777216.0f);
+        K += 24;
+    }
+    const uint32_t add = SR ? (h << (q.d - 16)) : (q.rtn_add + ((m >> q.d) & q.lsb_mask));
+    const uint32_t m2 = m + add;
+    const int f_pre = (int)(m >> 23) - K;                // E + E_max before rounding
+    const int f_post = (int)(m2 >> 23) - K;              // ... after a possible carry
+    uint32_t code = ((uint32_t)f_post << q.n1) | ((m2 >> q.d) & q.man_mask);
+    if (f_post >= q.nfield) code = q.top;                // E >= E_max: clip
+    if (f_pre <= 0 || mag == 0u) {                       // E <= -E_max: underflow
+        code = 0u;
+        if (SR && mag != 0u && a >= __fmul_rn(q.alpha, eps)) code = q.min_code;
+    }
+    return code ? (code | ((xb >> 31) ? q.sign_bit : 0u)) : 0u;
 }
 
 // Quantise one tile and write its slice of the packed stream.  Each lane packs
@@ -411,7 +438,7 @@ __device__ __forceinline__ uint32_t quant_elem(uint32_t xb, uint32_t addend, flo
 // `total_words` = words in the whole stream.
 template <int DT, int NBITS, bool SR, bool FAST, bool FULL>
 __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint64_t tile_base, uint64_t n,
-                                           uint64_t total_words, const QuantParams &q, uint64_t seed) {
+                                           uint64_t total_words, const QuantParams &q, uint64_t seed, const Weyl &wy) {
     constexpr int C = ElemTraits<DT>::kChunk;
     constexpr int B = C * NBITS;                           // bits per lane per load step: 32..128
     constexpr int NW = (B + 31) / 32;                      // words that hold a lane's bits
@@ -435,11 +462,11 @@ __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint6
             #pragma unroll
             for (int b = 0; b < C / 8; ++b) {
                 uint4 r = make_uint4(0u, 0u, 0u, 0u);
-                if (SR) r = rand_block(seed, (i >> 3) + b);
+                if (SR) r = rand_block(seed, (i >> 3) + b, wy);
                 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const int k = b * 8 + e;
-                    const uint32_t code = quant_elem<SR, FAST>(elem_bits<DT>(v[j], k), SR ? sr_addend(r, e, q.d) : 0u,
+                    const uint32_t code = quant_elem<SR, FAST>(elem_bits<DT>(v[j], k), SR ? rand_h(r, e) : 0u,
                                                                SR ? eps_of(r, e) : 0.f, q);
                     const int pos = k * NBITS;             // a constant once the loops are unrolled
                     cw[pos >> 5] |= code << (pos & 31);
