@@ -199,6 +199,35 @@ lgn_status lgn_compress_layers(const lgn_layer_t *layers, int num_layers,
                                lgn_layer_result_t *results_dev,
                                void *ws, size_t ws_bytes, void *stream);
 
+/* Statistics pass that needs no workspace from the caller.  (The paper has no
+ * counterpart: this is a convenience of the library, not a step of the method.)
+ *
+ * Same result as lgn_stats, bit for bit.  It is meant for callers that cannot
+ * allocate device memory at the point of the call: a hook that runs in the
+ * middle of a training step, where cudaMalloc would synchronise the whole
+ * device; a process that gave all free device memory to its own pool at start-up,
+ * so that a later cudaMalloc fails; a C or C++ plug-in that has no access to the
+ * host framework's allocator.  Such a caller still owns g and out_dev, but the
+ * kernel's scratch (queue header, descriptors, per-tile partial sums) lives in
+ * an array of LGN_STATS_STATIC_SCRATCH_BYTES bytes that is part of the library
+ * image: every GPU that loads the library holds it from load to process exit.
+ *   g, n, dt, out_dev, stream   as for lgn_stats
+ *   n above LGN_STATS_STATIC_MAX_ELEMS returns LGN_ERR_UNSUPPORTED (nothing is
+ *   enqueued); use lgn_stats with a caller workspace for larger tensors.
+ * The call itself allocates nothing on the device, neither directly nor through
+ * a library.  The first call on each device looks up the array's device address
+ * (one cudaGetSymbolAddress, with that device current) and remembers it; make
+ * that first call before starting any stream capture.
+ * All calls on one device share the one array: it still holds the previous
+ * call's contents when the next call starts (the call re-initialises what it
+ * reads), and two calls whose kernels can overlap on the GPU -- different
+ * streams without an ordering between them -- race on it and give wrong
+ * statistics.  Calls on one stream, or ordered by events, are safe. */
+#define LGN_STATS_STATIC_MAX_ELEMS      (1ull << 28)
+#define LGN_STATS_STATIC_SCRATCH_BYTES  (1024u + 32u * (1u << 14))
+lgn_status lgn_stats_static_scratch(const void *g, uint64_t n, lgn_dtype dt, lgn_stats_t *out_dev,
+                                    void *stream);
+
 /* The grouped path for tensors that live in HOST memory: copies every input to
  * the device, runs lgn_compress_layers, copies every output and the results
  * back, and waits for the stream.  This is the end-to-end form of the call a

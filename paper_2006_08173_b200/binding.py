@@ -80,6 +80,9 @@ _lib.lgn_compress_layers_host.argtypes = [C.POINTER(LayerT), _i32, C.POINTER(Lay
 _lib.lgn_compress_layers_host.restype = _i32
 _lib.lgn_launches_per_call.argtypes = [_i32]
 _lib.lgn_launches_per_call.restype = _i32
+_lib.lgn_stats_static_scratch.argtypes = [_vp, _u64, _i32, _vp, _vp]
+_lib.lgn_stats_static_scratch.restype = _i32
+STATS_STATIC_MAX_ELEMS = 1 << 28
 
 
 class LgnError(RuntimeError):
@@ -164,6 +167,14 @@ def lgn_stats_async(g: torch.Tensor, out_dev: torch.Tensor, ws: torch.Tensor, st
     """Enqueue the statistics pass; ``out_dev`` (>= 48 bytes, uint8, CUDA) receives one lgn_stats_t."""
     _check(_lib.lgn_stats(_dev(g, "g"), g.numel(), dtype_code(g), _dev(out_dev, "out_dev"),
                           _dev(ws, "ws"), ws.numel() * ws.element_size(), _stream(stream)), "lgn_stats")
+
+
+def lgn_stats_static_scratch_async(g: torch.Tensor, out_dev: torch.Tensor, stream=None) -> None:
+    """lgn_stats without a workspace argument: the scratch is an array inside
+    the library (at most STATS_STATIC_MAX_ELEMS elements; calls that may overlap
+    on the GPU must not share a device).  Allocates nothing."""
+    _check(_lib.lgn_stats_static_scratch(_dev(g, "g") if g.numel() else None, g.numel(), dtype_code(g),
+                                         _dev(out_dev, "out_dev"), _stream(stream)), "lgn_stats_static_scratch")
 
 
 def read_stats(out_dev: torch.Tensor) -> Dict[str, float]:

@@ -817,3 +817,44 @@ extern "C" lgn_status lgn_compress_layers_host(const lgn_layer_t *layers, int nu
         return LGN_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
 }
+
+// ------------------------------------------------------------------ statistics without a caller workspace
+// Scratch of lgn_stats_static_scratch: part of the library image on every device
+// that loads it.  In host code this name is only a handle for the symbol, not an
+// address a kernel can use: the device address comes from cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_stats_static_scratch[LGN_STATS_STATIC_SCRATCH_BYTES];
+
+namespace {
+// Device address of the array on the current device, looked up once per device.
+void *static_scratch_address() {
+    static void *cached[64];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (cached[dev] == nullptr) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_stats_static_scratch) != cudaSuccess) return nullptr;
+        cached[dev] = p;
+    }
+    return cached[dev];
+}
+}  // namespace
+
+extern "C" lgn_status lgn_stats_static_scratch(const void *g, uint64_t n, lgn_dtype dt, lgn_stats_t *out_dev,
+                                               void *stream) {
+    if (out_dev == nullptr || !aligned16(out_dev)) return LGN_ERR_INVALID_ARG;
+    if (n > LGN_STATS_STATIC_MAX_ELEMS) return LGN_ERR_UNSUPPORTED;
+    WsLayout w;
+    if (!ws_layout(&n, 1, w) || w.total > sizeof(g_stats_static_scratch)) return LGN_ERR_UNSUPPORTED;
+    InternalLayer il;
+    memset(&il, 0, sizeof il);
+    il.d.g = g; il.d.n = n; il.d.dt = dt; il.d.mode = kModeStatsOnly;
+    il.stats_out = out_dev;
+    lgn_status s = check_layer(il.d);                 // argument errors before touching CUDA
+    if (s != LGN_OK) return s;
+    void *scratch = static_scratch_address();
+    if (scratch == nullptr) return LGN_ERR_CUDA;
+    // run_layers rewrites the queue header, descriptors and counters on the stream
+    // before the kernel reads them; partial sums are written before they are read.
+    return run_layers(std::vector<InternalLayer>(1, il), scratch, sizeof(g_stats_static_scratch),
+                      static_cast<cudaStream_t>(stream));
+}
