@@ -1,0 +1,75 @@
+"""The bench workload at its full size (ResNet-18 shapes, batch 256, fp32,
+635.8 M elements, per-layer sparsity), in the launch configuration bench.py
+times: one lgn_compress_layers call over all 20 layers.  Statistics of every
+layer are compared with the oracle's over the whole tensor; outputs are compared
+bit for bit on sampled windows of every layer (and in full on the small layers)
+with the oracle's mu/sigma fed in; properties that hold at any size are checked
+over every element on the device."""
+import numpy as np
+import pytest
+import torch
+
+import bench
+from gpu_helpers import assert_stats_close, np_bits
+from paper_2006_08173_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def launch(lgn, w, specs, tensors, overrides=None):
+    outs = [torch.empty_like(g) for g in tensors]
+    layers = []
+    for k, (g, o, s) in enumerate(zip(tensors, outs, specs)):
+        ov = overrides[k] if overrides else (None, None)
+        layers.append(lgn.make_layer(g, o, lgn.MODE_PRUNE, S=s.sparsity, seed=1000 + k,
+                                     mu_override=ov[0], sigma_override=ov[1]))
+    ws = lgn.new_workspace([g.numel() for g in tensors], tensors[0].device)
+    res = lgn.new_results(len(tensors), tensors[0].device)
+    lgn.lgn_compress_layers(layers, res, ws)
+    torch.cuda.synchronize()
+    return outs, lgn.read_results(res, len(tensors))
+
+
+def test_bench_workload_full_size(lgn, oracle):
+    w, specs = bench.workload_specs("resnet18_bs256_fp32_prune", 256, 0)
+    tensors = synth.make_layers(specs, torch.float32, "cuda")
+    assert sum(t.numel() for t in tensors) == 635_830_272
+
+    # (a) free-running: statistics of every layer against the oracle over the whole tensor
+    outs, res = launch(lgn, w, specs, tensors)
+    ref_stats = []
+    for g, r in zip(tensors, res):
+        st = oracle.stats(np_bits(g))
+        ref_stats.append(st)
+        assert r["status"] == 0
+        assert_stats_close(r, st)
+    # properties over every element, on the device
+    for g, o, r, s in zip(tensors, outs, res, specs):
+        tau = r["tau"]
+        a = g.abs()
+        assert bool(torch.equal(o[a > tau], g[a > tau]))                         # above alpha: unchanged
+        small = a <= tau
+        vals = o[small]
+        assert bool(((vals == 0) | (vals.abs() == tau)).all())                   # else 0 or +-alpha
+        keep = small & (o != 0)
+        assert bool((torch.sign(o[keep]) == torch.sign(g[keep])).all())
+        achieved = float((o == 0).sum()) / o.numel()
+        assert abs(achieved - s.sparsity) < 1e-3 + 5 * (s.sparsity * (1 - s.sparsity) / o.numel()) ** 0.5
+
+    # (b) oracle's mu/sigma fed in: thresholds identical, outputs bit-exact on samples
+    ov = [(st["mu"], st["sigma"]) for st in ref_stats]
+    outs, res = launch(lgn, w, specs, tensors, overrides=ov)
+    rs = np.random.RandomState(0)
+    for k, (g, o, r, s, st) in enumerate(zip(tensors, outs, res, specs, ref_stats)):
+        tau = oracle.snap_tau(oracle.threshold(st["mu"], st["sigma"], st["zero_frac"], s.sparsity), oracle.F32)
+        assert r["tau"] == tau
+        n = g.numel()
+        if n <= 7_000_000:
+            windows = [(0, n)]                                                    # the small layers in full
+        else:
+            windows = [(0, 40_000), (n - 40_000, n)] + \
+                      [(int(x), int(x) + 40_000) for x in rs.randint(0, n - 40_000, 3)]
+        for lo, hi in windows:
+            ref = oracle.prune(np_bits(g[lo:hi]), tau, 1000 + k, first=lo)
+            got = np_bits(o[lo:hi])
+            assert np.array_equal(got.view(np.uint32), ref.view(np.uint32)), (k, lo)
