@@ -24,7 +24,8 @@
  *  - Gradient tensors (g, and out of a pruning call) must be 32-byte aligned;
  *    code streams, workspaces and result arrays 16-byte aligned.  Input and
  *    output buffers must not overlap.
- *  - Inputs must be finite.  +0 and -0 both count as zero.
+ *  - Inputs must be finite, with magnitudes below 2^104 (about 2e31).  +0 and -0
+ *    both count as zero.
  *  - Argument errors are found on the host and returned before anything is
  *    enqueued.  A CUDA error at enqueue time is returned as LGN_ERR_CUDA.
  *  - Same inputs, seed and arguments give bitwise the same outputs and the same

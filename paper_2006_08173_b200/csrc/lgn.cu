@@ -298,7 +298,7 @@ constexpr int kAny = -1;                      // template value: decided per lay
 // the hot tile bodies are inlined and nothing else is compiled into the kernel;
 // kAny for all four is the general kernel for mixed groups.
 template <int DT, int MODE, int NBITS, int SR>
-__global__ void __launch_bounds__(kThreads, 4)
+__global__ void __launch_bounds__(kThreads, kMinCtas)
 compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Segment *segs,
                 int num_layers, uint32_t total_items, Partial *partials) {
     __shared__ double sm_red[3 * kWarps];
@@ -405,14 +405,14 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
 
 // ------------------------------------------------------------------ stand-alone apply kernels
 template <int DT>
-__global__ void __launch_bounds__(kThreads, 4)
+__global__ void __launch_bounds__(kThreads, kMinCtas)
 prune_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, float tau, uint64_t seed, Weyl wy) {
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)
         run_prune_tile<DT, true>(g, out, n, tile, tau, seed, wy);
 }
 
 template <int DT, int NBITS, int SR>
-__global__ void __launch_bounds__(kThreads, 4)
+__global__ void __launch_bounds__(kThreads, kMinCtas)
 quantize_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, const __grid_constant__ QuantParams q,
                 uint64_t seed, Weyl wy) {
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)

@@ -18,9 +18,24 @@
 
 namespace lgn {
 
-constexpr int kThreads   = 256;
+// Launch shape; the defaults are the measured optimum, the macros exist for sweeps.
+#ifndef LGN_THREADS
+#define LGN_THREADS 256
+#endif
+#ifndef LGN_TILE_ELEMS
+#define LGN_TILE_ELEMS 32768
+#endif
+#ifndef LGN_MIN_CTAS
+#define LGN_MIN_CTAS 4
+#endif
+#ifndef LGN_LOADS_IN_FLIGHT
+#define LGN_LOADS_IN_FLIGHT 4
+#endif
+constexpr int kThreads   = LGN_THREADS;
 constexpr int kWarps     = kThreads / 32;
-constexpr int kTileElems = 16384;
+constexpr int kTileElems = LGN_TILE_ELEMS;
+constexpr int kMinCtas   = LGN_MIN_CTAS;      // resident CTAs per SM the kernels are compiled for
+constexpr int kInFlight  = LGN_LOADS_IN_FLIGHT;   // 32-byte loads a thread issues before it uses the first
 
 template <int DT> struct ElemTraits;
 template <> struct ElemTraits<LGN_F32>  { static constexpr int kChunk = 8;  static constexpr int kBytes = 4; };
@@ -176,9 +191,15 @@ __device__ __forceinline__ float eps_of(const uint4 &r, int e) {
 }
 
 // ---------------------------------------------------------------- statistics
-__device__ __forceinline__ float lg2_approx(float a) {
+// log2 of a magnitude scaled by 2^24.  The scaling (an exact multiply) lifts
+// every fp32 subnormal into the normal range, so the single-instruction
+// flush-to-zero form of the hardware approximation can be used: zero gives -inf,
+// everything else log2|x| + 24.  Magnitudes must stay below 2^104 (the product
+// must not overflow).
+constexpr float kLogShift = 24.0f;
+__device__ __forceinline__ float lg2_scaled(float a) {
     float y;
-    asm("lg2.approx.f32 %0, %1;" : "=f"(y) : "f"(a));   // subnormal inputs are handled (no .ftz)
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(a * 16777216.0f));
     return y;
 }
 
@@ -187,7 +208,7 @@ struct StatsAcc {            // per thread, in log2 units
     unsigned long long cnt = 0;
 };
 
-// Adds one tile to the thread's accumulators.  y = log2|x| in fp32.  The sums
+// Adds one tile to the thread's accumulators.  y = log2|x| + 24 in fp32.  The sums
 // are taken of d = y - P, where the pivot P is the largest y in the first run
 // of this thread's elements that holds a nonzero: d stays of the order of the
 // spread of the data whatever its scale, so short fp32 runs of d and d^2 lose
@@ -199,7 +220,7 @@ template <int DT, bool FULL>
 __device__ __forceinline__ void stats_tile(const void *g, uint64_t tile_base, uint64_t n, StatsAcc &acc) {
     constexpr int C = ElemTraits<DT>::kChunk;
     constexpr int kLoads = kTileElems / (kThreads * C);   // 8 (fp32) or 4 (bf16)
-    constexpr int kGroup = 2;                             // 32-byte loads in flight per thread
+    constexpr int kGroup = kInFlight;                     // 32-byte loads in flight per thread
     const float kUnset = -__int_as_float(0x7F800000);     // -inf: no nonzero seen yet
     float P = kUnset;
     double D1 = 0.0, D2 = 0.0;
@@ -216,7 +237,7 @@ __device__ __forceinline__ void stats_tile(const void *g, uint64_t tile_base, ui
             #pragma unroll
             for (int e = 0; e < 16; ++e) {
                 const int idx = r * 16 + e;
-                y[e] = lg2_approx(fabsf(u2f(elem_bits<DT>(v[idx / C], idx % C))));   // -inf for zero
+                y[e] = lg2_scaled(fabsf(u2f(elem_bits<DT>(v[idx / C], idx % C))));   // -inf for zero
             }
             if (P == kUnset) {
                 #pragma unroll
@@ -239,7 +260,7 @@ __device__ __forceinline__ void stats_tile(const void *g, uint64_t tile_base, ui
         }
     }
     if (Cn) {
-        const double p = (double)P, c = (double)Cn;
+        const double p = (double)P - (double)kLogShift, c = (double)Cn;   // pivot in true log2 units
         acc.s1 += D1 + c * p;
         acc.s2 += D2 + p * (2.0 * D1 + c * p);
         acc.cnt += Cn;
@@ -293,7 +314,7 @@ __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t ti
                                            float tau, uint64_t seed, const Weyl &wy) {
     constexpr int C = ElemTraits<DT>::kChunk;
     constexpr int kLoads = kTileElems / (kThreads * C);
-    constexpr int kGroup = 2;
+    constexpr int kGroup = kInFlight;
     constexpr bool ZCHECK = !FULL;                        // the general body also serves tiny thresholds
     #pragma unroll 1
     for (int j0 = 0; j0 < kLoads; j0 += kGroup) {
@@ -443,7 +464,7 @@ __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint6
     constexpr int B = C * NBITS;                           // bits per lane per load step: 32..128
     constexpr int NW = (B + 31) / 32;                      // words that hold a lane's bits
     constexpr int kLoads = kTileElems / (kThreads * C);
-    constexpr int kGroup = 2;
+    constexpr int kGroup = kInFlight;
     const int lane = threadIdx.x & 31;
     const int o0 = (B % 32 == 0) ? 0 : ((32 - ((lane * B) & 31)) & 31);   // first word boundary inside this lane
 
