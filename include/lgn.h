@@ -148,9 +148,7 @@ lgn_status lgn_prune(const void *g, void *out, uint64_t n, lgn_dtype dt, double 
  *   seed   as in lgn_prune; used only with LGN_ROUND_STOCHASTIC
  * With x' = x / 2^scale_exp = M * 2^E, E_max = 2^(exp_bits-1):
  *   E >= E_max  (before rounding) -> largest code;
- *   E <= -E_max (before rounding) -> 0 (nearest) or, stochastic, pruned by Eq. 5
- *                with alpha = the smallest normal 2^(1-E_max+scale_exp) and the same
- *                eps_i: the smallest normal if |x| >= fl32(alpha*eps_i), else 0;
+ *   E <= -E_max (before rounding) -> 0, under both roundings;
  *   else M rounded to man_bits (nearest: ties to the even mantissa; stochastic:
  *   h_i/2^16 of one mantissa step added, then truncated),
  *   a carry out of M moves to E, and E reaching E_max gives the largest code.

@@ -363,12 +363,8 @@ enum { ORC_ROUND_NEAREST = 0, ORC_ROUND_STOCHASTIC = 1 };
  *   E >= E_max  -> clipped.  2^E_max itself is not on the grid of a format
  *                  that also has to hold zero, so the clip value is the
  *                  largest code: exponent field 2^n2 - 1, mantissa all ones.
- *   E <= -E_max -> 0 under round-to-nearest.  Under stochastic rounding the
- *                  value is pruned by Eq. 5 with alpha = the smallest normal
- *                  (in the tensor's own units, 2^(1-E_max+e_s) as an fp32
- *                  number) and eps = (h+1)/2^16: it becomes the smallest normal
- *                  if |x| >= fl32(alpha*eps) and 0 otherwise, exactly as
- *                  orc_prune_one decides.
+ *   E <= -E_max -> 0, as printed, under both roundings ("these tiny
+ *                  gradients can be pruned", Section 4.4).
  *   otherwise   -> M is rounded to n1 fraction bits (step Delta = 2^-n1).
  *                  Nearest: ties to even.  Stochastic: h/2^16 of one step is
  *                  added and the sum is truncated.  M_q = 2 carries into E; if that reaches E_max
@@ -389,13 +385,7 @@ uint32_t orc_quantize_one(double x, int n2, int n1, int e_s, int rounding, uint3
     int E = ex - 1;
 
     if (E >= Emax) return sign | top;
-    if (E <= -Emax) {
-        if (rounding != ORC_ROUND_STOCHASTIC) return 0;
-        float alpha = (float)ldexp(1.0, 1 - Emax + e_s);             /* exact, or 0 / inf out of fp32 range */
-        double eps = (double)((h & 0xFFFFu) + 1u) / 65536.0;
-        double thr = (double)(float)((double)alpha * eps);
-        return (fabs(x) >= thr) ? (sign | (1u << n1)) : 0u;
-    }
+    if (E <= -Emax) return 0;
     double steps = (M - 1.0) * ldexp(1.0, n1);           /* exact: M has <= 23 fraction bits */
     double m;
     if (rounding == ORC_ROUND_STOCHASTIC) {

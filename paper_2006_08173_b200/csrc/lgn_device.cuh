@@ -95,8 +95,8 @@ __device__ __forceinline__ void st4_stream(void *p, uint32_t v) {
 template <int DT, bool FULL, Ld P>
 __device__ __forceinline__ Chunk load_chunk(const void *g, uint64_t i, uint64_t n) {
     constexpr int C = ElemTraits<DT>::kChunk;
-    if (FULL || i + C <= n)
-        return ld32<P, FULL>(static_cast<const char *>(g) + i * ElemTraits<DT>::kBytes);
+    if constexpr (FULL) return ld32<P, true>(static_cast<const char *>(g) + i * ElemTraits<DT>::kBytes);
+    if (i + C <= n) return ld32<P, false>(static_cast<const char *>(g) + i * ElemTraits<DT>::kBytes);
     Chunk c;
     #pragma unroll
     for (int k = 0; k < 8; ++k) c.w[k] = 0u;
@@ -398,21 +398,20 @@ __host__ __device__ inline QuantParams make_quant_params(const lgn_fp_format_t &
 // Code of one element from its fp32 bit pattern, integer arithmetic on the
 // pattern: adding the rounding increment below the kept bits lets a mantissa
 // carry run into the exponent field by itself.  h = the element's 16 random
-// bits, eps = (h+1)/2^16 (both unused for round-to-nearest).
+// bits (unused for round-to-nearest).
 //
 // FAST (K >= 1, the usual case: the layer scale is not so small that fp32
 // subnormal inputs could land inside the format's range).  With the pattern
 // taken as a signed integer and K << 23 subtracted, the arithmetic shift by d
 // gives [E + E_max | mantissa] directly; it is <= min_code exactly for the
 // values that underflow (E <= -E_max) and > top exactly for those that clip, so
-// one clamp to [min_code, top] settles both, and a value that underflows is
-// then either zeroed or left at min_code (stochastic survival, Eq. 5 with
-// alpha = the smallest normal).  The additions are written as multiply-adds
+// one clamp to [min_code, top] settles both, and a value that underflows
+// (|x| below the smallest normal) is then zeroed.  The additions are written as multiply-adds
 // with the run-time operand q.one so that they issue on the multiply-add pipe
 // and leave the integer ALU, the bottleneck of this kernel, to the shifts,
 // clamps and selects.
 template <bool SR, bool FAST>
-__device__ __forceinline__ uint32_t quant_elem(uint32_t xb, uint32_t h, float eps, const QuantParams &q) {
+__device__ __forceinline__ uint32_t quant_elem(uint32_t xb, uint32_t h, const QuantParams &q) {
     const uint32_t mag = xb & 0x7FFFFFFFu;
     const float a = u2f(mag);
     if (FAST) {
@@ -427,8 +426,7 @@ __device__ __forceinline__ uint32_t quant_elem(uint32_t xb, uint32_t h, float ep
         }
         const int raw = m2 >> q.d;                                        // arithmetic shift
         const uint32_t code = (uint32_t)min(max(raw, (int)q.min_code), (int)q.top);
-        bool kill = a < q.alpha;                                          // E <= -E_max: underflow
-        if (SR) kill = kill && (a < __fmul_rn(q.alpha, eps));             // ... unless it survives
+        const bool kill = a < q.alpha;                                    // E <= -E_max: underflow
         const uint32_t comb = (xb >> 31) * q.sign_bit + code;
         return kill ? 0u : comb;
     }
@@ -444,10 +442,7 @@ __device__ __forceinline__ uint32_t quant_elem(uint32_t xb, uint32_t h, float ep
     const int f_post = (int)(m2 >> 23) - K;              // ... after a possible carry
     uint32_t code = ((uint32_t)f_post << q.n1) | ((m2 >> q.d) & q.man_mask);
     if (f_post >= q.nfield) code = q.top;                // E >= E_max: clip
-    if (f_pre <= 0 || mag == 0u) {                       // E <= -E_max: underflow
-        code = 0u;
-        if (SR && mag != 0u && a >= __fmul_rn(q.alpha, eps)) code = q.min_code;
-    }
+    if (f_pre <= 0 || mag == 0u) code = 0u;              // E <= -E_max: underflow
     return code ? (code | ((xb >> 31) ? q.sign_bit : 0u)) : 0u;
 }
 
@@ -487,8 +482,7 @@ __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint6
                 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const int k = b * 8 + e;
-                    const uint32_t code = quant_elem<SR, FAST>(elem_bits<DT>(v[j], k), SR ? rand_h(r, e) : 0u,
-                                                               SR ? eps_of(r, e) : 0.f, q);
+                    const uint32_t code = quant_elem<SR, FAST>(elem_bits<DT>(v[j], k), SR ? rand_h(r, e) : 0u, q);
                     const int pos = k * NBITS;             // a constant once the loops are unrolled
                     cw[pos >> 5] |= code << (pos & 31);
                     if ((pos & 31) + NBITS > 32) cw[(pos >> 5) + 1] |= code >> (32 - (pos & 31));

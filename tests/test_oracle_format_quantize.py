@@ -209,47 +209,34 @@ def test_stochastic_rounding_probabilities_are_exact(oracle):
             assert step == 2.0 ** -n1
 
 
-def test_stochastic_underflow_is_eq5_with_the_smallest_normal(oracle):
-    """Below the smallest normal, stochastic rounding decides exactly as
-    stochastic pruning with alpha = the smallest normal does."""
+def test_underflow_flushes_under_both_roundings(oracle):
+    """Eq. 2 as printed: E <= -E_max gives 0, whatever the rounding mode and the
+    random bits; the smallest normal itself is kept."""
     for n2, n1, e_s in [(4, 1, 0), (5, 0, -17), (3, 2, -140), (2, 3, 5)]:
         Emax = 2 ** (n2 - 1)
         mn = 2.0 ** (1 - Emax + e_s)
         one = 1 << n1
-        sign = 1 << (n1 + n2)
-        rs = np.random.RandomState(n2)
-        for frac in [0.3, 0.75, 2.0 ** -10, 0.999999, 2.0 ** -17, 0.5] + list(rs.uniform(0, 1, 20)):
+        for frac in (0.999999, 0.75, 0.5, 2.0 ** -10):
             x = float(np.float32(mn * frac))
             if x == 0.0 or x >= mn:
                 continue
-            for h in [0, 1, 0x7FFF, 0x8000, 0xFFFE, 0xFFFF] + list(rs.randint(0, 65536, 40)):
-                want = oracle.prune_one(x, float(np.float32(mn)), int(h))
-                assert want in (0.0, float(np.float32(mn)))
-                got = oracle.quantize_one(x, n2, n1, e_s, SR, int(h))
-                assert got == (one if want != 0.0 else 0)
-                assert oracle.quantize_one(-x, n2, n1, e_s, SR, int(h)) == ((one | sign) if want != 0.0 else 0)
+            for h in (0, 1, 0x8000, 0xFFFF):
+                assert oracle.quantize_one(x, n2, n1, e_s, SR, h) == 0
+                assert oracle.quantize_one(-x, n2, n1, e_s, SR, h) == 0
             assert oracle.quantize_one(x, n2, n1, e_s, RTN, 0) == 0
-        # probability of surviving = |x| / smallest normal, to 16 bits (where fp32 can
-        # resolve alpha*eps: not when the smallest normal is itself an fp32 subnormal)
-        if mn < 2.0 ** -100:
-            continue
-        x = float(np.float32(mn * 0.3))
-        hits = sum(oracle.quantize_one(x, n2, n1, e_s, SR, h) != 0 for h in range(0, 65536, 7))
-        assert abs(hits / len(range(0, 65536, 7)) - x / mn) < 2e-3
-    assert oracle.quantize_one(2.0 ** -7 * 2.0 ** -30, 4, 1, 0, SR, 1) == 0
-    assert oracle.quantize_one(2.0 ** -7 * 2.0 ** -16, 4, 1, 0, SR, 0) == 2       # eps = 2^-16 exactly reached
+        for h in (0, 0xFFFF):
+            assert oracle.quantize_one(mn, n2, n1, e_s, SR, h) == one
 
 
 def test_stochastic_rounding_is_unbiased(oracle):
     rs = np.random.RandomState(3)
     n = 400_000
     n2, n1, e_s = 4, 1, -17
-    x = (2.0 ** rs.uniform(-12 + e_s, 6 + e_s, n)).astype(np.float32)      # spans underflow and range
+    x = (2.0 ** rs.uniform(-7 + e_s, 6 + e_s, n)).astype(np.float32)       # inside the range: E in [-7, 6]
     codes = oracle.quantize(x, n2, n1, e_s, SR, seed=5)
     dec = np.array([oracle.decode(c, n2, n1, e_s) for c in range(64)])[codes]
     binade = 2.0 ** np.floor(np.log2(x.astype(np.float64)))
     step = np.maximum(binade * 2.0 ** -n1, 0)          # in range: one mantissa step
-    step = np.where(x < 2.0 ** (1 - 8 + e_s), 2.0 ** (1 - 8 + e_s), step)
     rel = (dec - x) / step                              # each term has variance <= 1/4
     assert abs(rel.mean()) < 4 * 0.5 / math.sqrt(n)
 
