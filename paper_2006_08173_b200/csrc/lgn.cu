@@ -494,12 +494,20 @@ static lgn_status check_layer(const lgn_layer_t &d) {
     return LGN_OK;
 }
 
-// Queue order: statistics of layer k+1 are placed between the statistics and the
-// apply tiles of layer k, so the closed form of layer k is evaluated while other
-// tiles stream; a layer's apply run walks its tiles from the last one read back to
-// the first, the order in which L2 still holds them.
+// Queue order.  A layer's apply tiles can start only once its statistics are
+// complete and its closed form (about 10 us on one thread) is published, so other
+// work is placed between the two: statistics runs of the following layers are
+// pulled forward until at least kLookaheadBytes of input lie between the end of
+// S(k) and the start of A(k) (one following layer always; more when layers are
+// small).  Large layers therefore go S(k) S(k+1) A(k) S(k+2) A(k+1) ..., and a run
+// of small layers has several statistics runs in flight, all of which still fit in
+// L2 when their apply runs come.  A layer's apply run walks its tiles from the last
+// one read back to the first, the order in which L2 still holds them.
+constexpr uint64_t kLookaheadBytes = 96ull << 20;
+
 static void build_queue(const std::vector<LayerState> &st, std::vector<Segment> &segs, uint32_t &total_items) {
     uint32_t item = 0;
+    uint64_t bytes = 0;                                    // input bytes of all runs emitted so far
     auto push = [&](uint32_t layer, uint32_t phase) {
         if (st[layer].ntiles == 0) return;
         if (phase == 1 && st[layer].mode == kModeStatsOnly) return;
@@ -509,13 +517,19 @@ static void build_queue(const std::vector<LayerState> &st, std::vector<Segment> 
         s.tile_begin = 0; s.reverse = phase;
         segs.push_back(s);
         item += s.ntiles;
+        bytes += st[layer].n * (st[layer].dt == LGN_BF16 ? 2u : 4u);
     };
     const uint32_t L = (uint32_t)st.size();
+    std::vector<uint64_t> bytes_after_stats(L, 0);
+    uint32_t next_s = 0;
     for (uint32_t k = 0; k < L; ++k) {
-        push(k, 0);
-        if (k > 0) push(k - 1, 1);
+        while (next_s < L && (next_s <= k + 1 || bytes - bytes_after_stats[k] < kLookaheadBytes)) {
+            push(next_s, 0);
+            bytes_after_stats[next_s] = bytes;
+            ++next_s;
+        }
+        push(k, 1);
     }
-    if (L > 0) push(L - 1, 1);
     total_items = item;
 }
 
