@@ -139,6 +139,33 @@ __device__ __forceinline__ uint32_t elem_bits(const Chunk &c, int k) {
     return (k & 1) ? (c.w[k >> 1] & 0xFFFF0000u) : (c.w[k >> 1] << 16);
 }
 
+// Software-pipelined walk over a tile's load steps: two register buffers of
+// kGroup chunks each; the loads of the next group are issued before the current
+// group is processed, so a thread always has loads in flight while it computes.
+// body(buf, j) processes the kGroup chunks of load steps j .. j+kGroup-1.
+template <int DT, bool FULL, Ld P, int kLoads, int kGroup, class Body>
+__device__ __forceinline__ void pipelined_tile(const void *g, uint64_t tile_base, uint64_t n, Body body) {
+    constexpr int C = ElemTraits<DT>::kChunk;
+    static_assert(kLoads % (2 * kGroup) == 0, "load steps come in pairs of groups");
+    Chunk a[kGroup], b[kGroup];
+    #pragma unroll
+    for (int j = 0; j < kGroup; ++j)
+        a[j] = load_chunk<DT, FULL, P>(g, tile_base + (uint64_t)(j * kThreads + threadIdx.x) * C, n);
+    #pragma unroll 1
+    for (int j0 = 0; j0 < kLoads; j0 += 2 * kGroup) {
+        #pragma unroll
+        for (int j = 0; j < kGroup; ++j)
+            b[j] = load_chunk<DT, FULL, P>(g, tile_base + (uint64_t)((j0 + kGroup + j) * kThreads + threadIdx.x) * C, n);
+        body(a, j0);
+        if (j0 + 2 * kGroup < kLoads) {
+            #pragma unroll
+            for (int j = 0; j < kGroup; ++j)
+                a[j] = load_chunk<DT, FULL, P>(g, tile_base + (uint64_t)((j0 + 2 * kGroup + j) * kThreads + threadIdx.x) * C, n);
+        }
+        body(b, j0 + kGroup);
+    }
+}
+
 // ---------------------------------------------------------------- random bits
 // Philox4x32 (Salmon et al., SC'11), seven rounds: each round is two 32x32->64
 // multiplies with the halves crossed and xored with the counter and a
@@ -220,17 +247,12 @@ template <int DT, bool FULL>
 __device__ __forceinline__ void stats_tile(const void *g, uint64_t tile_base, uint64_t n, StatsAcc &acc) {
     constexpr int C = ElemTraits<DT>::kChunk;
     constexpr int kLoads = kTileElems / (kThreads * C);   // 8 (fp32) or 4 (bf16)
-    constexpr int kGroup = kInFlight;                     // 32-byte loads in flight per thread
+    constexpr int kGroup = 16 / C;                        // chunks per register buffer (two buffers): one run of 16
     const float kUnset = -__int_as_float(0x7F800000);     // -inf: no nonzero seen yet
     float P = kUnset;
     double D1 = 0.0, D2 = 0.0;
     unsigned long long Cn = 0;
-    #pragma unroll 1
-    for (int j0 = 0; j0 < kLoads; j0 += kGroup) {
-        Chunk v[kGroup];
-        #pragma unroll
-        for (int j = 0; j < kGroup; ++j)
-            v[j] = load_chunk<DT, FULL, Ld::Keep>(g, tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * C, n);
+    pipelined_tile<DT, FULL, Ld::Keep, kLoads, kGroup>(g, tile_base, n, [&](const Chunk (&v)[kGroup], int) {
         #pragma unroll
         for (int r = 0; r < kGroup * C / 16; ++r) {       // runs of 16 elements
             float y[16];
@@ -258,7 +280,7 @@ __device__ __forceinline__ void stats_tile(const void *g, uint64_t tile_base, ui
             D2 += (double)s2;
             Cn += c;
         }
-    }
+    });
     if (Cn) {
         const double p = (double)P - (double)kLogShift, c = (double)Cn;   // pivot in true log2 units
         acc.s1 += D1 + c * p;
@@ -314,14 +336,9 @@ __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t ti
                                            float tau, uint64_t seed, const Weyl &wy) {
     constexpr int C = ElemTraits<DT>::kChunk;
     constexpr int kLoads = kTileElems / (kThreads * C);
-    constexpr int kGroup = kInFlight;
+    constexpr int kGroup = 1;                             // one chunk per buffer: the apply bodies need the registers
     constexpr bool ZCHECK = !FULL;                        // the general body also serves tiny thresholds
-    #pragma unroll 1
-    for (int j0 = 0; j0 < kLoads; j0 += kGroup) {
-        Chunk v[kGroup];
-        #pragma unroll
-        for (int j = 0; j < kGroup; ++j)
-            v[j] = load_chunk<DT, FULL, Ld::Stream>(g, tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * C, n);
+    pipelined_tile<DT, FULL, Ld::Stream, kLoads, kGroup>(g, tile_base, n, [&](const Chunk (&v)[kGroup], int j0) {
         #pragma unroll
         for (int j = 0; j < kGroup; ++j) {
             const uint64_t i = tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * C;
@@ -345,7 +362,7 @@ __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t ti
             }
             store_chunk<DT, FULL>(out, i, n, o);
         }
-    }
+    });
 }
 
 // ---------------------------------------------------------------- FP quantisation (Eq. 1-2, Algorithm 1)
@@ -459,16 +476,11 @@ __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint6
     constexpr int B = C * NBITS;                           // bits per lane per load step: 32..128
     constexpr int NW = (B + 31) / 32;                      // words that hold a lane's bits
     constexpr int kLoads = kTileElems / (kThreads * C);
-    constexpr int kGroup = kInFlight;
+    constexpr int kGroup = 1;
     const int lane = threadIdx.x & 31;
     const int o0 = (B % 32 == 0) ? 0 : ((32 - ((lane * B) & 31)) & 31);   // first word boundary inside this lane
 
-    #pragma unroll 1
-    for (int j0 = 0; j0 < kLoads; j0 += kGroup) {
-        Chunk v[kGroup];
-        #pragma unroll
-        for (int j = 0; j < kGroup; ++j)
-            v[j] = load_chunk<DT, FULL, Ld::Stream>(g, tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * C, n);
+    pipelined_tile<DT, FULL, Ld::Stream, kLoads, kGroup>(g, tile_base, n, [&](const Chunk (&v)[kGroup], int j0) {
         #pragma unroll
         for (int j = 0; j < kGroup; ++j) {
             const uint64_t i = tile_base + (uint64_t)((j0 + j) * kThreads + threadIdx.x) * C;
@@ -512,7 +524,7 @@ __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint6
                 }
             }
         }
-    }
+    });
 }
 
 }  // namespace lgn
