@@ -201,7 +201,7 @@ __device__ __forceinline__ void run_quant_tile(const void *g, void *out, uint64_
     const uint64_t base = (uint64_t)tile * kTileElems;
     const uint64_t total_words = (n * (uint64_t)NBITS + 31) >> 5;
     uint32_t *codes = static_cast<uint32_t *>(out);
-    if (INLINE_HOT && base + kTileElems <= n && q.K >= 1)
+    if (INLINE_HOT && base + kTileElems <= n && q.K >= 1 && q.K <= 255)
         quant_tile<DT, NBITS, SR, true, true>(g, codes, base, n, total_words, q, seed, wy);
     else
         quant_tile_general<DT, NBITS, SR>(g, codes, base, n, total_words, q, seed, wy);

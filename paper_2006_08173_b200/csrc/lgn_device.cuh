@@ -463,6 +463,56 @@ __device__ __forceinline__ uint32_t quant_elem(uint32_t xb, uint32_t h, const Qu
     return code ? (code | ((xb >> 31) ? q.sign_bit : 0u)) : 0u;
 }
 
+// bf16 fast path: two elements at a time, both halves of a 32-bit word, in
+// 16-bit lanes (the element's own bf16 pattern already holds sign, the same
+// 8-bit exponent field as fp32, and 7 fraction bits).  Same arithmetic as
+// quant_elem's fast path with d' = 7 - man_bits dropped bits: rounding increment
+// added below the kept bits, shift, subtract K << man_bits and clamp to
+// [min_code, top] with the packed 16-bit add-max / min instructions, zero the
+// lanes whose magnitude is below the smallest normal, merge the signs, and
+// return the two codes side by side (low element first).  Needs 1 <= K <= 255 so
+// that every lane value fits a signed 16-bit integer.
+struct PackedQuant {
+    uint32_t dq;        // 7 - man_bits
+    uint32_t add_a;     // stochastic: lane mask of the dq random bits; nearest: 2^(dq-1) - 1 in both lanes
+    uint32_t add_b;     // stochastic: 16 - dq (shift of the random word); nearest: lane mask of the kept LSB
+    uint32_t keep2;     // lane mask of the 16 - dq bits left after the shift
+    uint32_t neg_ks2;   // -(K << man_bits) in both lanes
+    uint32_t min2, top2;
+    uint32_t neg_lim2;  // -(((K + 1) << 7) - 1) in both lanes: adding it leaves >= 1 exactly when in range
+    uint32_t sign2;     // sign bit of a code in both lanes
+};
+
+template <bool SR>
+__device__ __forceinline__ PackedQuant make_packed_quant(const QuantParams &q) {
+    PackedQuant p;
+    const uint32_t rep = 0x00010001u;
+    p.dq = 7u - (uint32_t)q.n1;
+    if (SR) { p.add_a = ((1u << p.dq) - 1u) * rep; p.add_b = 16u - p.dq; }
+    else    { p.add_a = ((1u << (p.dq - 1u)) - 1u) * rep; p.add_b = q.lsb_mask * rep; }
+    p.keep2 = ((1u << (16u - p.dq)) - 1u) * rep;
+    p.neg_ks2 = ((0u - ((uint32_t)q.K << q.n1)) & 0xFFFFu) * rep;
+    p.min2 = q.min_code * rep;
+    p.top2 = q.top * rep;
+    p.neg_lim2 = ((0u - ((((uint32_t)q.K + 1u) << 7) - 1u)) & 0xFFFFu) * rep;
+    p.sign2 = q.sign_bit * rep;
+    return p;
+}
+
+template <int NBITS, bool SR>
+__device__ __forceinline__ uint32_t quant_pair_bf16(uint32_t w, uint32_t r, const PackedQuant &p) {
+    const uint32_t mag2 = w & 0x7FFF7FFFu;
+    const uint32_t add2 = SR ? ((r >> p.add_b) & p.add_a) : (p.add_a + ((mag2 >> p.dq) & p.add_b));
+    const uint32_t m2 = mag2 + add2;                              // a finite lane cannot carry into its neighbour
+    const uint32_t post2 = (m2 >> p.dq) & p.keep2;                // [exponent field | mantissa] per lane
+    uint32_t c2 = __viaddmax_s16x2(post2, p.neg_ks2, p.min2);     // max(post - Ks, min_code)
+    c2 = __vmins2(c2, p.top2);
+    const uint32_t live2 = __vmins2(__viaddmax_s16x2(mag2, p.neg_lim2, 0u), 0x00010001u);   // 1 if in range, else 0
+    const uint32_t mask2 = live2 * 0xFFFFu;
+    const uint32_t fin2 = (c2 | ((w >> (16 - NBITS)) & p.sign2)) & mask2;
+    return (fin2 | (fin2 >> (16 - NBITS))) & ((1u << (2 * NBITS)) - 1u);
+}
+
 // Quantise one tile and write its slice of the packed stream.  Each lane packs
 // the codes of its chunk into B = kChunk*NBITS bits (up to four 32-bit words).
 // Output words are assembled from the lane in which they start and, where B is
@@ -479,6 +529,8 @@ __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint6
     constexpr int kGroup = 1;
     const int lane = threadIdx.x & 31;
     const int o0 = (B % 32 == 0) ? 0 : ((32 - ((lane * B) & 31)) & 31);   // first word boundary inside this lane
+    PackedQuant pq;
+    if constexpr (DT == LGN_BF16 && FAST) pq = make_packed_quant<SR>(q);
 
     pipelined_tile<DT, FULL, Ld::Stream, kLoads, kGroup>(g, tile_base, n, [&](const Chunk (&v)[kGroup], int j0) {
         #pragma unroll
@@ -491,13 +543,24 @@ __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint6
             for (int b = 0; b < C / 8; ++b) {
                 uint4 r = make_uint4(0u, 0u, 0u, 0u);
                 if (SR) r = rand_block(seed, (i >> 3) + b, wy);
-                #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int k = b * 8 + e;
-                    const uint32_t code = quant_elem<SR, FAST>(elem_bits<DT>(v[j], k), SR ? rand_h(r, e) : 0u, q);
-                    const int pos = k * NBITS;             // a constant once the loops are unrolled
-                    cw[pos >> 5] |= code << (pos & 31);
-                    if ((pos & 31) + NBITS > 32) cw[(pos >> 5) + 1] |= code >> (32 - (pos & 31));
+                if constexpr (DT == LGN_BF16 && FAST) {
+                    const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+                    #pragma unroll
+                    for (int pr = 0; pr < 4; ++pr) {       // word pr of the block <-> elements 2pr, 2pr+1
+                        const uint32_t two = quant_pair_bf16<NBITS, SR>(v[j].w[b * 4 + pr], rw[pr], pq);
+                        const int pos = (b * 8 + 2 * pr) * NBITS;
+                        cw[pos >> 5] |= two << (pos & 31);
+                        if ((pos & 31) + 2 * NBITS > 32) cw[(pos >> 5) + 1] |= two >> (32 - (pos & 31));
+                    }
+                } else {
+                    #pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const int k = b * 8 + e;
+                        const uint32_t code = quant_elem<SR, FAST>(elem_bits<DT>(v[j], k), SR ? rand_h(r, e) : 0u, q);
+                        const int pos = k * NBITS;         // a constant once the loops are unrolled
+                        cw[pos >> 5] |= code << (pos & 31);
+                        if ((pos & 31) + NBITS > 32) cw[(pos >> 5) + 1] |= code >> (32 - (pos & 31));
+                    }
                 }
             }
             const uint64_t lane_bit = i * (uint64_t)NBITS;  // position of this lane's bit 0 in the stream
