@@ -582,7 +582,7 @@ __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint6
                 for (int k = 0; k < NW; ++k) {
                     if (o0 + 32 * k < B) {
                         const uint32_t word = __funnelshift_r(s[k], s[k + 1], o0);
-                        if (w0 + k < total_words) st4_stream(codes + w0 + k, word);
+                        if (FULL || w0 + k < total_words) st4_stream(codes + w0 + k, word);   // a whole tile ends on a word boundary
                     }
                 }
             }
