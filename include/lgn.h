@@ -198,6 +198,19 @@ lgn_status lgn_compress_layers(const lgn_layer_t *layers, int num_layers,
                                lgn_layer_result_t *results_dev,
                                void *ws, size_t ws_bytes, void *stream);
 
+/* Self-test of the bounded device-side wait (no counterpart in the paper).
+ * Same arguments and the same work as lgn_compress_layers, except that one
+ * statistics tile of layer 0 is withheld from the queue, so layer 0's closed form
+ * is never published.  Every apply tile of layer 0 must give up after the bounded
+ * wait (about a second) instead of spinning for ever: the kernel ends,
+ * results_dev[0].status becomes LGN_ERR_TIMEOUT (its output is not written), the
+ * other layers complete normally, and the CUDA context stays usable.  results_dev
+ * must be zero-filled by the caller (layer 0's record is otherwise untouched).
+ * Nothing faults, traps or hangs.  layers[0].n must be > 0. */
+lgn_status lgn_selftest_wait_expires(const lgn_layer_t *layers, int num_layers,
+                                     lgn_layer_result_t *results_dev,
+                                     void *ws, size_t ws_bytes, void *stream);
+
 /* Statistics pass that needs no workspace from the caller.  (The paper has no
  * counterpart: this is a convenience of the library, not a step of the method.)
  *

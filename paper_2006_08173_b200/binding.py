@@ -78,6 +78,8 @@ _lib.lgn_host_staging_bytes.argtypes = [C.POINTER(LayerT), _i32]
 _lib.lgn_host_staging_bytes.restype = _sz
 _lib.lgn_compress_layers_host.argtypes = [C.POINTER(LayerT), _i32, C.POINTER(LayerResultT), _vp, _sz, _vp]
 _lib.lgn_compress_layers_host.restype = _i32
+_lib.lgn_selftest_wait_expires.argtypes = [C.POINTER(LayerT), _i32, _vp, _vp, _sz, _vp]
+_lib.lgn_selftest_wait_expires.restype = _i32
 _lib.lgn_launches_per_call.argtypes = [_i32]
 _lib.lgn_launches_per_call.restype = _i32
 _lib.lgn_stats_static_scratch.argtypes = [_vp, _u64, _i32, _vp, _vp]
@@ -231,6 +233,17 @@ def lgn_compress_layers(layers: Sequence[LayerT], results_dev: torch.Tensor, ws:
         raise ValueError("results_dev too small")
     _check(_lib.lgn_compress_layers(arr, L, _dev(results_dev, "results_dev"), _dev(ws, "ws"),
                                     ws.numel() * ws.element_size(), _stream(stream)), "lgn_compress_layers")
+
+
+def lgn_selftest_wait_expires(layers: Sequence[LayerT], results_dev: torch.Tensor, ws: torch.Tensor,
+                              stream=None) -> None:
+    """lgn_compress_layers with one statistics tile of layer 0 withheld: layer 0
+    must come back with status LGN_ERR_TIMEOUT after about a second."""
+    L = len(layers)
+    arr = (LayerT * max(1, L))(*layers)
+    _check(_lib.lgn_selftest_wait_expires(arr, L, _dev(results_dev, "results_dev"), _dev(ws, "ws"),
+                                          ws.numel() * ws.element_size(), _stream(stream)),
+           "lgn_selftest_wait_expires")
 
 
 def new_results(num_layers: int, device) -> torch.Tensor:
