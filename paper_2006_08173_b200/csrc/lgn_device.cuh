@@ -466,20 +466,22 @@ __device__ __forceinline__ uint32_t quant_elem(uint32_t xb, uint32_t h, const Qu
 // bf16 fast path: two elements at a time, both halves of a 32-bit word, in
 // 16-bit lanes (the element's own bf16 pattern already holds sign, the same
 // 8-bit exponent field as fp32, and 7 fraction bits).  Same arithmetic as
-// quant_elem's fast path with d' = 7 - man_bits dropped bits: rounding increment
-// added below the kept bits, shift, subtract K << man_bits and clamp to
-// [min_code, top] with the packed 16-bit add-max / min instructions, zero the
-// lanes whose magnitude is below the smallest normal, merge the signs, and
-// return the two codes side by side (low element first).  Needs 1 <= K <= 255 so
-// that every lane value fits a signed 16-bit integer.
+// quant_elem's fast path with d' = 7 - man_bits dropped bits, but measured from
+// the smallest normal: with lim = (K+1) << 7 (its bf16 pattern) and
+// t = magnitude - lim, a lane is below the smallest normal exactly when t < 0,
+// and otherwise its code is ((t + increment) >> d') + min_code, clipped to top
+// (lim is a multiple of 2^d', so this equals the shifted sum minus K << man_bits).
+// The packed 16-bit add-max / add-min instructions keep the lanes apart; the
+// lanes with t < 0 are zeroed by a byte permute that spreads each lane's sign
+// bit over the lane.  Needs 1 <= K <= 255 so that every lane value fits a signed
+// 16-bit integer.
 struct PackedQuant {
     uint32_t dq;        // 7 - man_bits
     uint32_t add_a;     // stochastic: lane mask of the dq random bits; nearest: 2^(dq-1) - 1 in both lanes
     uint32_t add_b;     // stochastic: 16 - dq (shift of the random word); nearest: lane mask of the kept LSB
     uint32_t keep2;     // lane mask of the 16 - dq bits left after the shift
-    uint32_t neg_ks2;   // -(K << man_bits) in both lanes
     uint32_t min2, top2;
-    uint32_t neg_lim2;  // -(((K + 1) << 7) - 1) in both lanes: adding it leaves >= 1 exactly when in range
+    uint32_t neg_lim2;  // -((K + 1) << 7) in both lanes
     uint32_t sign2;     // sign bit of a code in both lanes
 };
 
@@ -491,25 +493,31 @@ __device__ __forceinline__ PackedQuant make_packed_quant(const QuantParams &q) {
     if (SR) { p.add_a = ((1u << p.dq) - 1u) * rep; p.add_b = 16u - p.dq; }
     else    { p.add_a = ((1u << (p.dq - 1u)) - 1u) * rep; p.add_b = q.lsb_mask * rep; }
     p.keep2 = ((1u << (16u - p.dq)) - 1u) * rep;
-    p.neg_ks2 = ((0u - ((uint32_t)q.K << q.n1)) & 0xFFFFu) * rep;
     p.min2 = q.min_code * rep;
     p.top2 = q.top * rep;
-    p.neg_lim2 = ((0u - ((((uint32_t)q.K + 1u) << 7) - 1u)) & 0xFFFFu) * rep;
+    p.neg_lim2 = ((0u - (((uint32_t)q.K + 1u) << 7)) & 0xFFFFu) * rep;
     p.sign2 = q.sign_bit * rep;
     return p;
 }
 
+// 0xFFFF in every 16-bit lane whose sign bit is set, 0 elsewhere.
+__device__ __forceinline__ uint32_t lane_sign_mask(uint32_t x) {
+    uint32_t m;
+    asm("prmt.b32 %0, %1, %1, 0xBB99;" : "=r"(m) : "r"(x));   // bytes 1,1,3,3 with the sign-replicate flag
+    return m;
+}
+
 template <int NBITS, bool SR>
 __device__ __forceinline__ uint32_t quant_pair_bf16(uint32_t w, uint32_t r, const PackedQuant &p) {
+    const uint32_t none = 0x80008000u;                            // a max() against it changes nothing
     const uint32_t mag2 = w & 0x7FFF7FFFu;
-    const uint32_t add2 = SR ? ((r >> p.add_b) & p.add_a) : (p.add_a + ((mag2 >> p.dq) & p.add_b));
-    const uint32_t m2 = mag2 + add2;                              // a finite lane cannot carry into its neighbour
-    const uint32_t post2 = (m2 >> p.dq) & p.keep2;                // [exponent field | mantissa] per lane
-    uint32_t c2 = __viaddmax_s16x2(post2, p.neg_ks2, p.min2);     // max(post - Ks, min_code)
-    c2 = __vmins2(c2, p.top2);
-    const uint32_t live2 = __vmins2(__viaddmax_s16x2(mag2, p.neg_lim2, 0u), 0x00010001u);   // 1 if in range, else 0
-    const uint32_t mask2 = live2 * 0xFFFFu;
-    const uint32_t fin2 = (c2 | ((w >> (16 - NBITS)) & p.sign2)) & mask2;
+    const uint32_t t2 = __viaddmax_s16x2(mag2, p.neg_lim2, none); // magnitude - lim per lane, in [-32768, 32511]
+    const uint32_t add2 = SR ? ((r >> p.add_b) & p.add_a) : (p.add_a + ((t2 >> p.dq) & p.add_b));
+    const uint32_t m2 = __viaddmax_s16x2(t2, add2, none);         // per lane: no carry from a negative lane
+    const uint32_t post2 = (m2 >> p.dq) & p.keep2;                // [exponent field - (K+1) | mantissa] per lane
+    const uint32_t c2 = __viaddmin_s16x2(post2, p.min2, p.top2);  // min(post + min_code, top)
+    const uint32_t dead2 = lane_sign_mask(t2);
+    const uint32_t fin2 = (c2 | ((w >> (16 - NBITS)) & p.sign2)) & ~dead2;
     return (fin2 | (fin2 >> (16 - NBITS))) & ((1u << (2 * NBITS)) - 1u);
 }
 
