@@ -183,7 +183,7 @@ template <int DT, bool INLINE_HOT>
 __device__ __forceinline__ void run_prune_tile(const void *g, void *out, uint64_t n, uint32_t tile,
                                                float tau, uint64_t seed, const Weyl &wy) {
     const uint64_t base = (uint64_t)tile * kTileElems;
-    const bool tiny = tau > 0.f && tau < 1.17549435e-38f;     // alpha*eps could round to zero
+    const bool tiny = tau > 0.f && tau < kPruneFastMin;       // alpha*2^-16 inexact, or alpha*eps could round to zero
     if (INLINE_HOT && base + kTileElems <= n && !tiny) prune_tile<DT, true>(g, out, base, n, tau, seed, wy);
     else                                               prune_tile_general<DT>(g, out, base, n, tau, seed, wy);
 }

@@ -330,7 +330,36 @@ __device__ __forceinline__ uint32_t prune_elem(uint32_t xb, float eps, float tau
     return p ? kept : 0u;
 }
 
-// tau == 0 never reaches this function (the caller copies the tile instead).
+// Hot-path forms, for alpha >= kPruneFastMin.  c = alpha * 2^-16 is then exact, and
+// fma(h, c, c) = fl32(c * (h + 1)) = fl32(alpha * eps): the same single rounding as
+// above with one instruction less.
+constexpr float kPruneFastMin = 0x1p-100f;
+
+__device__ __forceinline__ uint32_t prune_elem_fast(uint32_t xb, float hf, float c, float tau) {
+    const float a = fabsf(u2f(xb));
+    const float thr = fmaf(hf, c, c);
+    const uint32_t kept = (xb & 0x80000000u) | f2u(fmaxf(a, tau));
+    return a >= thr ? kept : 0u;
+}
+
+// bf16, two elements of one 32-bit word at a time.  A bf16 magnitude a (pattern
+// a16) and a non-negative fp32 threshold (pattern tb) compare as their patterns:
+// a >= thr  <=>  (a16 << 16) >= tb  <=>  (a16 << 16) - tb >= 0 as a signed integer
+// (both are below 2^31).  The two differences' sign bits, spread over their 16-bit
+// lanes by one byte permute, zero the pruned lanes; max(a, alpha) is a packed
+// 16-bit maximum because alpha is a bf16 value too.
+__device__ __forceinline__ uint32_t prune_pair_bf16(uint32_t w, uint32_t r, float c, uint32_t tau2) {
+    const float h0 = (float)(unsigned short)(r & 0xFFFFu), h1 = (float)(unsigned short)(r >> 16);
+    const uint32_t mag2 = w & 0x7FFF7FFFu;
+    const uint32_t d0 = (mag2 << 16) - f2u(fmaf(h0, c, c));
+    const uint32_t d1 = (mag2 & 0xFFFF0000u) - f2u(fmaf(h1, c, c));
+    uint32_t dead2;
+    asm("prmt.b32 %0, %1, %2, 0xFFBB;" : "=r"(dead2) : "r"(d0), "r"(d1));   // sign of d0 | sign of d1, per lane
+    const uint32_t kept2 = __vmaxs2(mag2, tau2) | (w & 0x80008000u);
+    return kept2 & ~dead2;
+}
+
+// tau == 0 never reaches the fast forms' arithmetic (the tile is copied instead).
 template <int DT, bool FULL>
 __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t tile_base, uint64_t n,
                                            float tau, uint64_t seed, const Weyl &wy) {
@@ -338,6 +367,8 @@ __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t ti
     constexpr int kLoads = kTileElems / (kThreads * C);
     constexpr int kGroup = 1;                             // one chunk per buffer: the apply bodies need the registers
     constexpr bool ZCHECK = !FULL;                        // the general body also serves tiny thresholds
+    const float c = tau * 0x1p-16f;                       // used by the hot path only (FULL: alpha >= kPruneFastMin or 0)
+    const uint32_t tau2 = (f2u(tau) >> 16) * 0x00010001u; // alpha's bf16 pattern in both lanes
     pipelined_tile<DT, FULL, Ld::Stream, kLoads, kGroup>(g, tile_base, n, [&](const Chunk (&v)[kGroup], int j0) {
         #pragma unroll
         for (int j = 0; j < kGroup; ++j) {
@@ -350,13 +381,21 @@ __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t ti
                 #pragma unroll
                 for (int b = 0; b < C / 8; ++b) {
                     const uint4 r = rand_block(seed, (i >> 3) + b, wy);
-                    #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const int k = b * 8 + e;
-                        const uint32_t res = prune_elem<ZCHECK>(elem_bits<DT>(v[j], k), eps_of(r, e), tau);
-                        if (DT == LGN_F32) o.w[k] = res;
-                        else if ((k & 1) == 0) o.w[k >> 1] = res >> 16;
-                        else o.w[k >> 1] |= res & 0xFFFF0000u;
+                    if constexpr (FULL && DT == LGN_BF16) {
+                        const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+                        #pragma unroll
+                        for (int pr = 0; pr < 4; ++pr) o.w[b * 4 + pr] = prune_pair_bf16(v[j].w[b * 4 + pr], rw[pr], c, tau2);
+                    } else {
+                        #pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const int k = b * 8 + e;
+                            uint32_t res;
+                            if constexpr (FULL) res = prune_elem_fast(elem_bits<DT>(v[j], k), rand_hf(r, e), c, tau);
+                            else                res = prune_elem<ZCHECK>(elem_bits<DT>(v[j], k), eps_of(r, e), tau);
+                            if (DT == LGN_F32) o.w[k] = res;
+                            else if ((k & 1) == 0) o.w[k >> 1] = res >> 16;
+                            else o.w[k >> 1] |= res & 0xFFFF0000u;
+                        }
                     }
                 }
             }
