@@ -84,6 +84,16 @@ def _L():
         lib.orc_unpack.argtypes = [vp, u64, i32, vp]
         lib.orc_unpack.restype = None
         lib.orc_count_zeros.argtypes = [vp, u64, i32]
+        lib.orc_prefix_blocks.argtypes = [u64]
+        lib.orc_prefix_blocks.restype = u64
+        lib.orc_prefix_bound_words.argtypes = [u64, i32]
+        lib.orc_prefix_bound_words.restype = u64
+        lib.orc_prefix_class.argtypes = [u32, i32, dbl]
+        lib.orc_prefix_class.restype = i32
+        lib.orc_prefix_encode.argtypes = [vp, u64, i32, dbl, vp, vp]
+        lib.orc_prefix_encode.restype = u64
+        lib.orc_prefix_decode.argtypes = [vp, vp, u64, i32, dbl, vp]
+        lib.orc_prefix_decode.restype = None
         lib.orc_count_zeros.restype = u64
         _lib = lib
     return _lib
@@ -238,3 +248,40 @@ def unpack(packed: np.ndarray, n: int, nbits: int) -> np.ndarray:
 def count_zeros(g: np.ndarray) -> int:
     g = _flat(g)
     return int(_L().orc_count_zeros(_ptr(g), g.size, _dtype_of(g)))
+
+
+# --------------------------------------------------------------------------- prefix code (appendix "Encoding")
+PREFIX_BLOCK = 2048
+
+
+def prefix_blocks(n: int) -> int:
+    return int(_L().orc_prefix_blocks(n))
+
+
+def prefix_bound_words(n: int, dtype: int) -> int:
+    return int(_L().orc_prefix_bound_words(n, dtype))
+
+
+def prefix_class(pattern: int, dtype: int, tau_used: float) -> int:
+    """0 zero, 1 +alpha, 2 -alpha, 3 FP value."""
+    return int(_L().orc_prefix_class(pattern, dtype, tau_used))
+
+
+def prefix_encode(v: np.ndarray, tau_used: float):
+    """(stream uint32[words], off uint64[nblocks+1]) of a pruned tensor."""
+    v = _flat(v)
+    dt = _dtype_of(v)
+    stream = np.zeros(max(1, prefix_bound_words(v.size, dt)), dtype=np.uint32)
+    off = np.zeros(prefix_blocks(v.size) + 1, dtype=np.uint64)
+    words = int(_L().orc_prefix_encode(_ptr(v), v.size, dt, tau_used, _ptr(stream), _ptr(off)))
+    return stream[:words].copy(), off
+
+
+def prefix_decode(stream: np.ndarray, off: np.ndarray, n: int, dtype: int, tau_used: float) -> np.ndarray:
+    stream = np.ascontiguousarray(stream, dtype=np.uint32)
+    off = np.ascontiguousarray(off, dtype=np.uint64)
+    if stream.size == 0:
+        stream = np.zeros(1, dtype=np.uint32)
+    out = np.empty(n, dtype=np.uint16 if dtype == BF16 else np.float32)
+    _L().orc_prefix_decode(_ptr(stream), _ptr(off), n, dtype, tau_used, _ptr(out))
+    return out

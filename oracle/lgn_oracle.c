@@ -24,6 +24,9 @@
  *                      derivation of Eq. 4; Monte-Carlo with orc_quantize
  *   orc_quantize_*     brute force over every code of every format
  *   orc_philox4x32     known-answer vectors published with the generator (10 rounds)
+ *   orc_prefix_*       the code table of the paper's appendix written out by hand for a
+ *                      worked example; decode(encode(x)) == x; length = n0 + 3 n_alpha +
+ *                      (2 + width) n_fp; the paper's "4 bits at 80 %, 2 bits at 90 %"
  *   end-to-end tensors parity unpinned by the paper (it prints no worked
  *                      numeric example of a compressed tensor)
  *
@@ -466,4 +469,112 @@ uint64_t orc_count_zeros(const void *g, uint64_t n, int dtype)
     uint64_t z = 0;
     for (uint64_t i = 0; i < n; ++i) z += (elem(g, dtype, i) == 0.0);
     return z;
+}
+
+/* ------------------------------------------------------------------ */
+/* Appendix "Encoding": prefix code for stochastically pruned tensors   */
+/* ------------------------------------------------------------------ */
+
+/* The paper's table gives the code words: 0 -> "0", +alpha -> "100",
+ * -alpha -> "101", anything else -> "11" followed by the FP value.  It fixes
+ * neither a bit order nor a container, so the stream format is this
+ * repository's (the CUDA library states the same format in its header):
+ *   - code words are emitted left to right as printed; the FP value follows
+ *     "11" as the element's own bit pattern (32 bits fp32, 16 bits bf16),
+ *     least-significant bit first;
+ *   - stream bit k is bit (k mod 32) of 32-bit word (k div 32);
+ *   - elements are taken in index order in blocks of 2048; block b starts at
+ *     word off[b], is padded with zero bits to a whole word, and off[nblocks]
+ *     is the length of the stream in words;
+ *   - "0" is the pattern of +0 only (a -0 travels as an FP value, so that the
+ *     code is lossless); the alpha codes exist only when alpha > 0. */
+#define ORC_PREFIX_BLOCK 2048u
+
+uint64_t orc_prefix_blocks(uint64_t n) { return (n + ORC_PREFIX_BLOCK - 1) / ORC_PREFIX_BLOCK; }
+
+/* worst case: every element an FP value */
+uint64_t orc_prefix_bound_words(uint64_t n, int dtype)
+{
+    uint64_t per = (dtype == ORC_BF16 ? 16u : 32u) + 2u;
+    uint64_t full = n / ORC_PREFIX_BLOCK, rest = n % ORC_PREFIX_BLOCK;
+    return full * ((ORC_PREFIX_BLOCK * per + 31) / 32) + (rest * per + 31) / 32;
+}
+
+static uint32_t pattern_of(const void *v, int dtype, uint64_t i)
+{
+    if (dtype == ORC_BF16) return ((const uint16_t *)v)[i];
+    uint32_t w; memcpy(&w, (const float *)v + i, sizeof w); return w;
+}
+
+static uint32_t tau_pattern(double tau_used, int dtype)
+{
+    float f = (float)tau_used; uint32_t w; memcpy(&w, &f, sizeof w);
+    return dtype == ORC_BF16 ? (w >> 16) : w;
+}
+
+/* 0: zero, 1: +alpha, 2: -alpha, 3: FP value */
+int orc_prefix_class(uint32_t pattern, int dtype, double tau_used)
+{
+    uint32_t sign = dtype == ORC_BF16 ? 0x8000u : 0x80000000u;
+    if (pattern == 0u) return 0;
+    if (tau_used > 0.0 && (pattern & ~sign) == tau_pattern(tau_used, dtype)) return (pattern & sign) ? 2 : 1;
+    return 3;
+}
+
+static void put_bit(uint32_t *stream, uint64_t *pos, int bit)
+{
+    if (bit) stream[*pos >> 5] |= 1u << (*pos & 31);
+    ++*pos;
+}
+
+static int get_bit(const uint32_t *stream, uint64_t *pos)
+{
+    int b = (stream[*pos >> 5] >> (*pos & 31)) & 1u;
+    ++*pos;
+    return b;
+}
+
+/* stream must hold orc_prefix_bound_words(n) zero-initialised words; off holds nblocks+1 entries.
+ * Returns the stream length in words. */
+uint64_t orc_prefix_encode(const void *v, uint64_t n, int dtype, double tau_used,
+                           uint32_t *stream, uint64_t *off)
+{
+    int width = dtype == ORC_BF16 ? 16 : 32;
+    uint64_t pos = 0, b = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        if (i % ORC_PREFIX_BLOCK == 0) {
+            pos = (pos + 31) / 32 * 32;            /* pad the previous block to a whole word */
+            off[b++] = pos / 32;
+        }
+        uint32_t p = pattern_of(v, dtype, i);
+        switch (orc_prefix_class(p, dtype, tau_used)) {
+        case 0: put_bit(stream, &pos, 0); break;
+        case 1: put_bit(stream, &pos, 1); put_bit(stream, &pos, 0); put_bit(stream, &pos, 0); break;
+        case 2: put_bit(stream, &pos, 1); put_bit(stream, &pos, 0); put_bit(stream, &pos, 1); break;
+        default:
+            put_bit(stream, &pos, 1); put_bit(stream, &pos, 1);
+            for (int k = 0; k < width; ++k) put_bit(stream, &pos, (p >> k) & 1u);
+        }
+    }
+    pos = (pos + 31) / 32 * 32;
+    off[b] = pos / 32;
+    return pos / 32;
+}
+
+void orc_prefix_decode(const uint32_t *stream, const uint64_t *off, uint64_t n, int dtype,
+                       double tau_used, void *out)
+{
+    int width = dtype == ORC_BF16 ? 16 : 32;
+    uint32_t sign = dtype == ORC_BF16 ? 0x8000u : 0x80000000u;
+    uint32_t tp = tau_pattern(tau_used, dtype);
+    uint64_t pos = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        if (i % ORC_PREFIX_BLOCK == 0) pos = off[i / ORC_PREFIX_BLOCK] * 32;
+        uint32_t p;
+        if (!get_bit(stream, &pos)) p = 0u;
+        else if (!get_bit(stream, &pos)) p = get_bit(stream, &pos) ? (tp | sign) : tp;
+        else { p = 0u; for (int k = 0; k < width; ++k) p |= (uint32_t)get_bit(stream, &pos) << k; }
+        if (dtype == ORC_BF16) ((uint16_t *)out)[i] = (uint16_t)p;
+        else memcpy((float *)out + i, &p, sizeof p);
+    }
 }
