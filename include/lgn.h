@@ -198,6 +198,46 @@ lgn_status lgn_compress_layers(const lgn_layer_t *layers, int num_layers,
                                lgn_layer_result_t *results_dev,
                                void *ws, size_t ws_bytes, void *stream);
 
+/* ---- Prefix code for pruned tensors (the paper's appendix "Encoding") ----------
+ * Code words, emitted left to right: a zero -> "0", +alpha -> "100", -alpha ->
+ * "101", any other value -> "11" followed by the value itself.  The paper gives
+ * the table only; the container is this library's:
+ *   - elements in index order, in blocks of LGN_PREFIX_BLOCK; block b occupies the
+ *     32-bit words off[b] .. off[b+1]-1 of the stream (zero bits pad it to a whole
+ *     word); off[nblocks] is the stream length in words;
+ *   - stream bit k is bit (k mod 32) of word (k div 32);
+ *   - the value after "11" is the element's own bit pattern (32 bits fp32, 16 bits
+ *     bf16), least-significant bit first;
+ *   - "0" stands for the pattern of +0 only (a -0 travels as a value: the code is
+ *     lossless); the alpha codes are used only when alpha > 0.
+ * lgn_prefix_encode reads g (device, 32-byte aligned, n elements).  With
+ * apply_prune != 0 it first applies Eq. 5 with threshold alpha and `seed` to every
+ * element on the fly -- bit for bit what lgn_prune would have written -- so the
+ * dense pruned tensor never exists; with apply_prune == 0 g is taken as it is (an
+ * already pruned tensor).  alpha is `tau` (snapped to the tensor's type like
+ * lgn_prune does), or, if tau_from_dev is not NULL, the tau field of that
+ * device-resident layer result (so that the call can follow lgn_compress_layers on
+ * the same stream without a host round trip).
+ * Outputs (device): off_dev[0 .. lgn_prefix_blocks(n)] and stream_dev.  A block
+ * that would end beyond capacity_words is not written; the caller detects this
+ * as off_dev[nblocks] > capacity_words.  lgn_prefix_bound_words(n, dt) is the
+ * capacity that always suffices.  ws: device scratch of
+ * lgn_prefix_workspace_bytes(n) bytes, 16-byte aligned, free again when the call's
+ * work on `stream` has finished.  Errors: as for the other entry points; n above
+ * 2^34 is LGN_ERR_UNSUPPORTED.  Three launches, no allocation, no synchronisation.
+ * lgn_prefix_decode is the inverse: n elements of type dt into out_dev. */
+#define LGN_PREFIX_BLOCK 2048u
+uint64_t   lgn_prefix_blocks(uint64_t n);
+uint64_t   lgn_prefix_bound_words(uint64_t n, lgn_dtype dt);
+size_t     lgn_prefix_workspace_bytes(uint64_t n);
+lgn_status lgn_prefix_encode(const void *g, uint64_t n, lgn_dtype dt, double tau, uint64_t seed,
+                             int apply_prune, const lgn_layer_result_t *tau_from_dev,
+                             uint32_t *stream_dev, uint64_t capacity_words, uint64_t *off_dev,
+                             void *ws, size_t ws_bytes, void *stream);
+lgn_status lgn_prefix_decode(const uint32_t *stream_dev, const uint64_t *off_dev, uint64_t n, lgn_dtype dt,
+                             double tau, const lgn_layer_result_t *tau_from_dev, void *out_dev,
+                             void *stream);
+
 /* Self-test of the bounded device-side wait (no counterpart in the paper).
  * Same arguments and the same work as lgn_compress_layers, except that one
  * statistics tile of layer 0 is withheld from the queue, so layer 0's closed form

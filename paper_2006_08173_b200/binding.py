@@ -80,6 +80,16 @@ _lib.lgn_compress_layers_host.argtypes = [C.POINTER(LayerT), _i32, C.POINTER(Lay
 _lib.lgn_compress_layers_host.restype = _i32
 _lib.lgn_selftest_wait_expires.argtypes = [C.POINTER(LayerT), _i32, _vp, _vp, _sz, _vp]
 _lib.lgn_selftest_wait_expires.restype = _i32
+_lib.lgn_prefix_blocks.argtypes = [_u64]
+_lib.lgn_prefix_blocks.restype = _u64
+_lib.lgn_prefix_bound_words.argtypes = [_u64, _i32]
+_lib.lgn_prefix_bound_words.restype = _u64
+_lib.lgn_prefix_workspace_bytes.argtypes = [_u64]
+_lib.lgn_prefix_workspace_bytes.restype = _sz
+_lib.lgn_prefix_encode.argtypes = [_vp, _u64, _i32, C.c_double, _u64, _i32, _vp, _vp, _u64, _vp, _vp, _sz, _vp]
+_lib.lgn_prefix_encode.restype = _i32
+_lib.lgn_prefix_decode.argtypes = [_vp, _vp, _u64, _i32, C.c_double, _vp, _vp, _vp]
+_lib.lgn_prefix_decode.restype = _i32
 _lib.lgn_launches_per_call.argtypes = [_i32]
 _lib.lgn_launches_per_call.restype = _i32
 _lib.lgn_stats_static_scratch.argtypes = [_vp, _u64, _i32, _vp, _vp]
@@ -298,3 +308,44 @@ def lgn_compress_layers_host(layers: Sequence[LayerT], dev_buf: torch.Tensor, st
                                          dev_buf.numel() * dev_buf.element_size(), _stream(stream)),
            "lgn_compress_layers_host")
     return [_result_dict(res[k]) for k in range(L)]
+
+
+# --------------------------------------------------------------------------- prefix code (appendix "Encoding")
+PREFIX_BLOCK = 2048
+
+
+def lgn_prefix_blocks(n: int) -> int:
+    return int(_lib.lgn_prefix_blocks(n))
+
+
+def lgn_prefix_bound_words(n: int, dtype_code_: int) -> int:
+    return int(_lib.lgn_prefix_bound_words(n, dtype_code_))
+
+
+def lgn_prefix_workspace_bytes(n: int) -> int:
+    return int(_lib.lgn_prefix_workspace_bytes(n))
+
+
+def lgn_prefix_encode(g: torch.Tensor, tau: float, seed: int, apply_prune: bool, stream_dev: torch.Tensor,
+                      off_dev: torch.Tensor, ws: torch.Tensor, tau_from_dev: Optional[int] = None,
+                      stream=None) -> None:
+    """``stream_dev``: int32/uint32 CUDA tensor (capacity = its length in words);
+    ``off_dev``: int64 CUDA tensor of lgn_prefix_blocks(n) + 1 entries;
+    ``tau_from_dev``: device address of a layer result record, or None."""
+    if off_dev.numel() < lgn_prefix_blocks(g.numel()) + 1 or off_dev.element_size() != 8:
+        raise ValueError("off_dev too small")
+    if stream_dev.element_size() != 4:
+        raise ValueError("stream_dev must hold 32-bit words")
+    _check(_lib.lgn_prefix_encode(_dev(g, "g") if g.numel() else None, g.numel(), dtype_code(g), float(tau), int(seed),
+                                  1 if apply_prune else 0, tau_from_dev,
+                                  _dev(stream_dev, "stream_dev") if stream_dev.numel() else None, stream_dev.numel(),
+                                  _dev(off_dev, "off_dev"), _dev(ws, "ws"), ws.numel() * ws.element_size(),
+                                  _stream(stream)), "lgn_prefix_encode")
+
+
+def lgn_prefix_decode(stream_dev: torch.Tensor, off_dev: torch.Tensor, out: torch.Tensor, tau: float,
+                      tau_from_dev: Optional[int] = None, stream=None) -> torch.Tensor:
+    _check(_lib.lgn_prefix_decode(_dev(stream_dev, "stream_dev") if stream_dev.numel() else None,
+                                  _dev(off_dev, "off_dev"), out.numel(), dtype_code(out), float(tau), tau_from_dev,
+                                  _dev(out, "out") if out.numel() else None, _stream(stream)), "lgn_prefix_decode")
+    return out
