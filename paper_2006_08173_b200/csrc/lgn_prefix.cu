@@ -71,11 +71,21 @@ __device__ __forceinline__ void pfx_values(uint32_t (&p)[kPfxPerThread], uint64_
                                            const Weyl &wy) {
     if (!PRUNE || tau == 0.f) return;
     const uint4 r = rand_block(seed, i >> 3, wy);
-    #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        const uint32_t xb = DT == LGN_F32 ? p[k] : p[k] << 16;
-        const uint32_t res = prune_elem<true>(xb, eps_of(r, k), tau);
-        p[k] = DT == LGN_F32 ? res : res >> 16;
+    if (tau >= kPruneFastMin) {                                   // same values, cheaper form (see prune_elem_fast)
+        const float c = tau * 0x1p-16f;
+        #pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t xb = DT == LGN_F32 ? p[k] : p[k] << 16;
+            const uint32_t res = prune_elem_fast(xb, rand_hf(r, k), c, tau);
+            p[k] = DT == LGN_F32 ? res : res >> 16;
+        }
+    } else {
+        #pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t xb = DT == LGN_F32 ? p[k] : p[k] << 16;
+            const uint32_t res = prune_elem<true>(xb, eps_of(r, k), tau);
+            p[k] = DT == LGN_F32 ? res : res >> 16;
+        }
     }
 }
 
@@ -98,61 +108,127 @@ template <int DT, bool PRUNE>
 __global__ void __launch_bounds__(kPfxThreads)
 prefix_count_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host, const lgn_layer_result_t *tau_from,
                     uint64_t seed, Weyl wy, uint32_t *block_words) {
-    __shared__ uint32_t sm[kPfxWarps];
+    __shared__ uint32_t sm_total[2];
     const float tau = pfx_tau(tau_host, tau_from);
     const uint32_t tp = tau_pattern<DT>(tau);
-    for (uint64_t b = blockIdx.x; b < nblocks; b += gridDim.x) {
+    if (threadIdx.x < 2) sm_total[threadIdx.x] = 0u;
+    __syncthreads();
+    uint32_t p[kPfxPerThread], q[kPfxPerThread];
+    uint64_t b = blockIdx.x;
+    if (b < nblocks) pfx_load<DT>(g, b * LGN_PREFIX_BLOCK + (uint64_t)threadIdx.x * kPfxPerThread, n, p);
+    for (uint32_t it = 0; b < nblocks; b += gridDim.x, ++it) {
         const uint64_t i = b * LGN_PREFIX_BLOCK + (uint64_t)threadIdx.x * kPfxPerThread;
-        uint32_t p[kPfxPerThread];
-        pfx_load<DT>(g, i, n, p);
+        const uint64_t bn = b + gridDim.x;                       // the next block's loads fly while this one is counted
+        if (bn < nblocks) pfx_load<DT>(g, bn * LGN_PREFIX_BLOCK + (uint64_t)threadIdx.x * kPfxPerThread, n, q);
         pfx_values<DT, PRUNE>(p, i, tau, seed, wy);
         uint32_t bits = 0u;
-        #pragma unroll
-        for (int k = 0; k < 8; ++k) if (i + k < n) bits += pfx_len<DT>(p[k], tp);
-        #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) bits += __shfl_down_sync(0xFFFFFFFFu, bits, off);
-        if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = bits;
+        if ((b + 1) * LGN_PREFIX_BLOCK <= n) {                   // the whole block lies inside the tensor
+            #pragma unroll
+            for (int k = 0; k < 8; ++k) bits += pfx_len<DT>(p[k], tp);
+        } else {
+            #pragma unroll
+            for (int k = 0; k < 8; ++k) if (i + k < n) bits += pfx_len<DT>(p[k], tp);
+        }
+        bits = __reduce_add_sync(0xFFFFFFFFu, bits);
+        if ((threadIdx.x & 31) == 0) atomicAdd(&sm_total[it & 1], bits);
         __syncthreads();
         if (threadIdx.x == 0) {
-            uint32_t t = 0u;
-            #pragma unroll
-            for (int w = 0; w < kPfxWarps; ++w) t += sm[w];
-            block_words[b] = (t + 31u) >> 5;
+            block_words[b] = (sm_total[it & 1] + 31u) >> 5;
+            sm_total[it & 1] = 0u;                               // used again two blocks on, after the next barrier
         }
-        __syncthreads();
+        #pragma unroll
+        for (int k = 0; k < 8; ++k) p[k] = q[k];
     }
 }
 
 // Exclusive prefix sum of block_words[0..nblocks) into off[0..nblocks]; one CTA.
+// Thread t owns the entries [t*per, (t+1)*per), per a multiple of 4 (16-byte loads).
 constexpr int kScanThreads = 1024;
 __global__ void __launch_bounds__(kScanThreads)
 prefix_scan_kernel(const uint32_t *block_words, uint64_t nblocks, uint64_t *off) {
-    __shared__ unsigned long long sm[kScanThreads];
-    const uint64_t per = (nblocks + kScanThreads - 1) / kScanThreads;
-    const uint64_t lo = (uint64_t)threadIdx.x * per;
+    __shared__ unsigned long long sm[kScanThreads / 32];
+    const uint64_t per = ((nblocks + kScanThreads - 1) / kScanThreads + 3) / 4 * 4;
+    const uint64_t lo = (uint64_t)threadIdx.x * per < nblocks ? (uint64_t)threadIdx.x * per : nblocks;
     const uint64_t hi = lo + per < nblocks ? lo + per : nblocks;
     unsigned long long s = 0;
-    for (uint64_t b = lo; b < hi; ++b) s += block_words[b];
-    sm[threadIdx.x] = s;
-    __syncthreads();
-    for (int d = 1; d < kScanThreads; d <<= 1) {                 // inclusive scan of the per-thread sums
-        unsigned long long v = threadIdx.x >= d ? sm[threadIdx.x - d] : 0ull;
-        __syncthreads();
-        sm[threadIdx.x] += v;
-        __syncthreads();
+    uint64_t k = lo;
+    for (; k + 4 <= hi; k += 4) {                                // lo is a multiple of 4: aligned
+        const uint4 v = *reinterpret_cast<const uint4 *>(block_words + k);
+        s += (unsigned long long)v.x + v.y + v.z + v.w;
     }
-    unsigned long long run = threadIdx.x ? sm[threadIdx.x - 1] : 0ull;
-    for (uint64_t b = lo; b < hi; ++b) { off[b] = run; run += block_words[b]; }
-    if (threadIdx.x == kScanThreads - 1) off[nblocks] = sm[kScanThreads - 1];
+    for (; k < hi; ++k) s += block_words[k];
+    // inclusive scan of s over the CTA: warp shuffles, then the 32 warp totals
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned long long incl = s;
+    #pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const unsigned long long v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += v;
+    }
+    if (lane == 31) sm[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned long long w = sm[lane];
+        #pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned long long v = __shfl_up_sync(0xFFFFFFFFu, w, d);
+            if (lane >= d) w += v;
+        }
+        sm[lane] = w;                                            // inclusive over warps
+    }
+    __syncthreads();
+    unsigned long long run = incl - s + (warp ? sm[warp - 1] : 0ull);
+    for (k = lo; k + 4 <= hi; k += 4) {
+        const uint4 v = *reinterpret_cast<const uint4 *>(block_words + k);
+        off[k] = run; off[k + 1] = run + v.x; off[k + 2] = run + v.x + v.y; off[k + 3] = run + v.x + v.y + v.z;
+        run += (unsigned long long)v.x + v.y + v.z + v.w;
+    }
+    for (; k < hi; ++k) { off[k] = run; run += block_words[k]; }
+    if (threadIdx.x == kScanThreads - 1) off[nblocks] = sm[kScanThreads / 32 - 1];
 }
 
 constexpr int kPfxImageWords = (LGN_PREFIX_BLOCK * 34u + 31u) / 32u + 2u;   // a block of FP values, plus slack
 
-// ORs `len` (<= 32) bits of v into the block image at bit position pos.
-__device__ __forceinline__ void pfx_put(uint32_t *img, uint32_t pos, uint32_t v, uint32_t len) {
-    const uint32_t w = pos >> 5, s = pos & 31u;
-    atomicOr(&img[w], v << s);
-    if (s + len > 32u) atomicOr(&img[w + 1], v >> (32u - s));
+// A thread's code words, assembled in a 64-bit register that starts at the
+// thread's bit position inside its first image word; every completed 32-bit word
+// is ORed into the image (the first and last word of a thread are shared with its
+// neighbours; words that are all zero -- runs of "0" codes -- need no write).
+// nvalid = how many of the 8 elements exist (8 except in the tensor's last block).
+template <int DT>
+__device__ __forceinline__ void pfx_emit_thread(const uint32_t (&p)[kPfxPerThread], uint32_t tp, uint32_t pos,
+                                                uint32_t nvalid, uint32_t *img) {
+    constexpr uint32_t kSign = PfxTraits<DT>::kSign;
+    // Two 32-bit registers hold the bits from the current image word on; `tot` is
+    // the thread's bit position in the image.  Written without branches (selects
+    // and a predicated shared-memory OR): the lanes of a warp would take different
+    // paths at almost every element otherwise.
+    const uint32_t img_addr = (uint32_t)__cvta_generic_to_shared(img);
+    uint32_t lo = 0u, hi = 0u, tot = pos;
+    auto append = [&](uint32_t x, uint32_t len) {                // x has `len` bits; the low register has room
+        const uint32_t s = tot & 31u;
+        lo |= x << s;
+        hi |= __funnelshift_l(x, 0u, s);                         // x >> (32 - s), and 0 for s = 0
+        const uint32_t after = tot + len;
+        const uint32_t full = (after ^ tot) & 32u;               // the low register's word is complete
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\tsetp.ne.and.u32 p, %1, 0, p;\n\t"
+                     "@p red.shared.or.b32 [%0], %1;\n\t}"
+                     :: "r"(img_addr + (tot >> 5) * 4u), "r"(lo), "r"(full) : "memory");
+        lo = full ? hi : lo;
+        hi = full ? 0u : hi;
+        tot = after;
+    };
+    #pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const bool in = (uint32_t)k < nvalid;
+        const uint32_t pat = p[k];
+        const bool zero = pat == 0u;
+        const bool alpha = tp != 0u && (pat & ~kSign) == tp;
+        const bool value = in && !zero && !alpha;
+        const uint32_t v = zero ? 0u : alpha ? ((pat & kSign) ? 5u : 1u) : 3u;       // first stream bit in bit 0
+        append(in ? v : 0u, !in ? 0u : zero ? 1u : alpha ? 3u : 2u);
+        append(value ? pat : 0u, value ? (uint32_t)PfxTraits<DT>::kWidth : 0u);
+    }
+    if (lo) atomicOr(&img[tot >> 5], lo);
 }
 
 template <int DT, bool PRUNE>
@@ -164,18 +240,27 @@ prefix_emit_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host, 
     const float tau = pfx_tau(tau_host, tau_from);
     const uint32_t tp = tau_pattern<DT>(tau);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t p[kPfxPerThread], q[kPfxPerThread];
+    if (blockIdx.x < nblocks)
+        pfx_load<DT>(g, (uint64_t)blockIdx.x * LGN_PREFIX_BLOCK + (uint64_t)threadIdx.x * kPfxPerThread, n, p);
     for (uint64_t b = blockIdx.x; b < nblocks; b += gridDim.x) {
         const uint64_t w0 = off[b], w1 = off[b + 1];
         const uint32_t words = (uint32_t)(w1 - w0);
-        if (w1 > capacity_words) continue;                       // does not fit: the caller sees off[nblocks] > capacity
-        for (uint32_t k = threadIdx.x; k < words + 1u; k += kPfxThreads) img[k] = 0u;
         const uint64_t i = b * LGN_PREFIX_BLOCK + (uint64_t)threadIdx.x * kPfxPerThread;
-        uint32_t p[kPfxPerThread];
-        pfx_load<DT>(g, i, n, p);
+        const uint64_t bn = b + gridDim.x;                       // the next block's loads fly while this one is packed
+        if (bn < nblocks) pfx_load<DT>(g, bn * LGN_PREFIX_BLOCK + (uint64_t)threadIdx.x * kPfxPerThread, n, q);
+        if (w1 > capacity_words) {                               // does not fit: the caller sees off[nblocks] > capacity
+            #pragma unroll
+            for (int k = 0; k < 8; ++k) p[k] = q[k];
+            continue;
+        }
+        for (uint32_t k = threadIdx.x; k < words + 1u; k += kPfxThreads) img[k] = 0u;
         pfx_values<DT, PRUNE>(p, i, tau, seed, wy);
-        uint32_t len[kPfxPerThread], bits = 0u;
+        const bool full = (b + 1) * LGN_PREFIX_BLOCK <= n;
+        const uint32_t nvalid = full ? 8u : (i >= n ? 0u : (n - i < 8u ? (uint32_t)(n - i) : 8u));
+        uint32_t bits = 0u;
         #pragma unroll
-        for (int k = 0; k < 8; ++k) { len[k] = i + k < n ? pfx_len<DT>(p[k], tp) : 0u; bits += len[k]; }
+        for (int k = 0; k < 8; ++k) if ((uint32_t)k < nvalid) bits += pfx_len<DT>(p[k], tp);
         // exclusive scan of `bits` over the CTA: warp scan, then the warp totals
         uint32_t incl = bits;
         #pragma unroll
@@ -188,21 +273,13 @@ prefix_emit_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host, 
         uint32_t pos = incl - bits;
         #pragma unroll
         for (int w = 0; w < kPfxWarps; ++w) if (w < warp) pos += sm[w];
-        #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            if (len[k] == 1u) {
-                // "0": the image is already zero there
-            } else if (len[k] == 3u) {
-                pfx_put(img, pos, (p[k] & PfxTraits<DT>::kSign) ? 5u : 1u, 3u);    // "101" / "100", first bit in bit 0
-            } else if (len[k] != 0u) {
-                pfx_put(img, pos, 3u, 2u);                                          // "11"
-                pfx_put(img, pos + 2u, p[k], PfxTraits<DT>::kWidth);
-            }
-            pos += len[k];
-        }
+        if (full) pfx_emit_thread<DT>(p, tp, pos, 8u, img);
+        else      pfx_emit_thread<DT>(p, tp, pos, nvalid, img);
         __syncthreads();
         for (uint32_t k = threadIdx.x; k < words; k += kPfxThreads) stream[w0 + k] = img[k];
         __syncthreads();                                         // the image and sm are reused by the next block
+        #pragma unroll
+        for (int k = 0; k < 8; ++k) p[k] = q[k];
     }
 }
 
@@ -245,11 +322,16 @@ prefix_decode_kernel(const uint32_t *stream, const uint64_t *off, uint64_t n, ui
 
 static bool aligned_to(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
-static int sm_count() {
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return -1;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
-    return sms;
+// Resident CTAs of a grid-stride kernel: SM count x CTAs per SM, at most one CTA per block of work.
+template <class K>
+static unsigned resident_grid(K kernel, uint64_t nblocks) {
+    int dev = 0, sms = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kPfxThreads, 0) != cudaSuccess) return 0;
+    if (per_sm < 1) per_sm = 1;
+    const uint64_t g = (uint64_t)sms * (uint64_t)per_sm;
+    return (unsigned)(nblocks < g ? nblocks : g);
 }
 
 }  // namespace lgn
@@ -285,18 +367,17 @@ extern "C" lgn_status lgn_prefix_encode(const void *g, uint64_t n, lgn_dtype dt,
     const float tau_used = dt == LGN_BF16 ? snap_threshold_bf16(tau) : snap_threshold_f32(tau);
     const Weyl wy = { kWeyl0, kWeyl1 };
     if (nb > 0) {
-        const int sms = sm_count();
-        if (sms < 1) return LGN_ERR_CUDA;
-        const unsigned grid = (unsigned)(nb < (uint64_t)sms * 8u ? nb : (uint64_t)sms * 8u);
+        #define LGN_PFX1(K, D, P, ...) { const unsigned grid = resident_grid(K<D, P>, nb); \
+                                         if (grid == 0) return LGN_ERR_CUDA; \
+                                         K<D, P><<<grid, kPfxThreads, 0, st>>>(__VA_ARGS__); }
         #define LGN_PFX(K, ...) \
-            if (dt == LGN_F32) { if (apply_prune) K<LGN_F32, true><<<grid, kPfxThreads, 0, st>>>(__VA_ARGS__); \
-                                 else             K<LGN_F32, false><<<grid, kPfxThreads, 0, st>>>(__VA_ARGS__); } \
-            else               { if (apply_prune) K<LGN_BF16, true><<<grid, kPfxThreads, 0, st>>>(__VA_ARGS__); \
-                                 else             K<LGN_BF16, false><<<grid, kPfxThreads, 0, st>>>(__VA_ARGS__); }
+            if (dt == LGN_F32) { if (apply_prune) LGN_PFX1(K, LGN_F32, true, __VA_ARGS__) else LGN_PFX1(K, LGN_F32, false, __VA_ARGS__) } \
+            else               { if (apply_prune) LGN_PFX1(K, LGN_BF16, true, __VA_ARGS__) else LGN_PFX1(K, LGN_BF16, false, __VA_ARGS__) }
         LGN_PFX(prefix_count_kernel, g, n, nb, tau_used, tau_from_dev, seed, wy, bw)
         prefix_scan_kernel<<<1, kScanThreads, 0, st>>>(bw, nb, off_dev);
         LGN_PFX(prefix_emit_kernel, g, n, nb, tau_used, tau_from_dev, seed, wy, off_dev, stream_dev, capacity_words)
         #undef LGN_PFX
+        #undef LGN_PFX1
     } else {
         prefix_scan_kernel<<<1, kScanThreads, 0, st>>>(bw, 0, off_dev);
     }
