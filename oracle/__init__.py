@@ -84,6 +84,8 @@ def _L():
         lib.orc_unpack.argtypes = [vp, u64, i32, vp]
         lib.orc_unpack.restype = None
         lib.orc_count_zeros.argtypes = [vp, u64, i32]
+        lib.orc_dequantize.argtypes = [vp, u64, i32, i32, i32, i32, i32, vp]
+        lib.orc_dequantize.restype = None
         lib.orc_prefix_blocks.argtypes = [u64]
         lib.orc_prefix_blocks.restype = u64
         lib.orc_prefix_bound_words.argtypes = [u64, i32]
@@ -284,4 +286,16 @@ def prefix_decode(stream: np.ndarray, off: np.ndarray, n: int, dtype: int, tau_u
         stream = np.zeros(1, dtype=np.uint32)
     out = np.empty(n, dtype=np.uint16 if dtype == BF16 else np.float32)
     _L().orc_prefix_decode(_ptr(stream), _ptr(off), n, dtype, tau_used, _ptr(out))
+    return out
+
+
+# --------------------------------------------------------------------------- decode of a packed stream (Algorithm 1)
+def dequantize(packed: np.ndarray, n: int, fmt: dict, out_dtype: int) -> np.ndarray:
+    """The tensor a packed code stream stands for, as float32 or bf16 bit patterns (uint16)."""
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    if packed.size == 0:
+        packed = np.zeros(1, dtype=np.uint8)
+    out = np.empty(n, dtype=np.uint16 if out_dtype == BF16 else np.float32)
+    _L().orc_dequantize(_ptr(packed), n, fmt["nbits"], fmt["exp_bits"], fmt["man_bits"], fmt["scale_exp"],
+                        out_dtype, _ptr(out))
     return out

@@ -24,6 +24,9 @@
  *                      derivation of Eq. 4; Monte-Carlo with orc_quantize
  *   orc_quantize_*     brute force over every code of every format
  *   orc_philox4x32     known-answer vectors published with the generator (10 rounds)
+ *   orc_dequantize     every code of every format against the value formula of Eq. 1-2
+ *                      written out in the test; quantising the decoded value (nearest)
+ *                      gives the code back
  *   orc_prefix_*       the code table of the paper's appendix written out by hand for a
  *                      worked example; decode(encode(x)) == x; length = n0 + 3 n_alpha +
  *                      (2 + width) n_fp; the paper's "4 bits at 80 %, 2 bits at 90 %"
@@ -576,5 +579,27 @@ void orc_prefix_decode(const uint32_t *stream, const uint64_t *off, uint64_t n, 
         else { p = 0u; for (int k = 0; k < width; ++k) p |= (uint32_t)get_bit(stream, &pos) << k; }
         if (dtype == ORC_BF16) ((uint16_t *)out)[i] = (uint16_t)p;
         else memcpy((float *)out + i, &p, sizeof p);
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* Algorithm 1, last step: the tensor a packed code stream stands for   */
+/* ------------------------------------------------------------------ */
+
+/* X_Q = 2^e_s * Q_FP(.) for every element of a packed stream: code i is bits
+ * [i*nbits, (i+1)*nbits) of the little-endian bit stream (orc_pack), decoded by
+ * orc_decode and stored in the output type.  Every decoded value has at most 7
+ * significant bits, so fp32 and bf16 hold it exactly whenever its exponent is in
+ * their normal range; the caller keeps formats inside that range. */
+void orc_dequantize(const uint8_t *packed, uint64_t n, int nbits, int n2, int n1, int e_s,
+                    int out_dtype, void *out)
+{
+    for (uint64_t i = 0; i < n; ++i) {
+        uint32_t code = 0;
+        for (int b = 0; b < nbits; ++b) {
+            uint64_t bit = i * (uint64_t)nbits + (uint64_t)b;
+            code |= (uint32_t)((packed[bit >> 3] >> (bit & 7)) & 1u) << b;
+        }
+        store_elem(out, out_dtype, i, orc_decode(code, n2, n1, e_s));
     }
 }
