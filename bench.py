@@ -57,6 +57,17 @@ for _dt in ("fp32", "bf16"):
                                                     mode="quant", nbits=6, rounding=1)
 
 
+# Steps next to the path (not bench lines: timed for the tables in profiles/):
+# the decoder of a packed code stream and the prefix-code encoder, on flat tensors.
+for _lg in (26, 28):
+    for _odt in ("fp32", "bf16"):
+        WORKLOADS[f"dequant_fp6_to_{_odt}_2p{_lg}"] = dict(net="aux", kind="dequant", log2n=_lg, nbits=6,
+                                                           dtype="f32" if _odt == "fp32" else "bf16", mode="dequant")
+    for _dt in ("fp32", "bf16"):
+        WORKLOADS[f"prefix_encode_{_dt}_2p{_lg}"] = dict(net="aux", kind="prefix", log2n=_lg,
+                                                         dtype="f32" if _dt == "fp32" else "bf16", mode="prefix")
+
+
 def workload_specs(name: str, batch: int, seed: int):
     w = WORKLOADS[name]
     if w["net"] == "resnet18":
@@ -325,6 +336,70 @@ def run_ours(args):
         print(json.dumps(line))
 
 
+def run_aux(args):
+    """Times one of the steps next to the path on a flat tensor (one GPU, no e2e / CPU legs)."""
+    from paper_2006_08173_b200 import binding as lgn
+    w = WORKLOADS[args.workload]
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    n = 1 << w["log2n"]
+    dtype = torch.float32 if w["dtype"] == "f32" else torch.bfloat16
+    esize = 4 if w["dtype"] == "f32" else 2
+    launches = 1
+    if w["kind"] == "dequant":
+        g = synth.lognormal_tensor(n, -12.0, 2.0, 0.5, 0, torch.bfloat16, str(dev))
+        st = lgn.lgn_stats(g)
+        fmt = lgn.lgn_fp_format(st["mu"], st["sigma"], w["nbits"])
+        codes = lgn.lgn_quantize(g, fmt, lgn.ROUND_STOCHASTIC, 1)
+        del g
+        out = torch.empty(n, dtype=dtype, device=dev)
+        alg_bytes = n * (w["nbits"] / 8.0 + esize)
+        call = lambda: lgn.lgn_dequantize(codes, n, fmt, out)
+        kernel = "dequantize_kernel"
+    else:
+        g = synth.lognormal_tensor(n, -12.0, 2.0, 0.5, 0, dtype, str(dev))
+        st = lgn.lgn_stats(g)
+        tau = lgn.lgn_threshold(st["mu"], st["sigma"], 1.0 - st["nnz"] / st["n"], 0.8)
+        stream_dev = torch.empty(lgn.lgn_prefix_bound_words(n, lgn.dtype_code(g)), dtype=torch.int32, device=dev)
+        off_dev = torch.empty(lgn.lgn_prefix_blocks(n) + 1, dtype=torch.int64, device=dev)
+        ws = torch.empty(max(16, lgn.lgn_prefix_workspace_bytes(n)), dtype=torch.uint8, device=dev)
+        call = lambda: lgn.lgn_prefix_encode(g, tau, 1, True, stream_dev, off_dev, ws)
+        call()
+        torch.cuda.synchronize()
+        words = int(off_dev[-1].item())
+        alg_bytes = n * esize + 4.0 * words          # one read of the tensor + the stream written
+        kernel = "prefix_count_kernel + prefix_scan_kernel + prefix_emit_kernel"
+        launches = 3
+    for _ in range(args.warmup):
+        call()
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    sampler = ClockSampler(0)
+    for i in range(args.steps):
+        starts[i].record(stream)
+        call()
+        ends[i].record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    per_step_ms = [a.elapsed_time(b) for a, b in zip(starts, ends)]
+    ms = statistics.mean(per_step_ms)
+    peak, peak_kind = read_peak()
+    achieved = alg_bytes / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": f"{w['kind']}_algorithmic_GBps", "value": achieved, "unit": "GB/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": w["dtype"], "data": "synthetic",
+        "config": {"workload": args.workload, "elements": n, "l2": "inputs and outputs larger than L2"},
+        "elements_per_s": n / (ms * 1e-3), "gpu_launches": args.steps * launches,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": kernel,
+                     "algorithmic_bytes_per_launch": alg_bytes, "best_ms": min(per_step_ms),
+                     "median_ms": statistics.median(per_step_ms)},
+        "clocks": clocks}))
+
+
 def lib_sha():
     import hashlib
     h = hashlib.sha1()
@@ -399,7 +474,11 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.impl == "reference":
+    if WORKLOADS[args.workload]["net"] == "aux":
+        if args.impl == "reference" or args.gpus != 1:
+            raise SystemExit("the auxiliary workloads are timed on one GPU by our arm only")
+        run_aux(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -238,6 +238,22 @@ lgn_status lgn_prefix_decode(const uint32_t *stream_dev, const uint64_t *off_dev
                              double tau, const lgn_layer_result_t *tau_from_dev, void *out_dev,
                              void *stream);
 
+/* ---- Decoder of a packed code stream (Algorithm 1, last step: X_Q = 2^e_s * Q_FP) ----
+ * What the consumer of a quantised gradient calls: code i of the stream written by
+ * lgn_quantize or lgn_compress_layers becomes element i of a dense fp32 or bf16
+ * tensor,  (-1)^s (1 + m / 2^man_bits) 2^(field - E_max + scale_exp)  for an
+ * exponent field != 0 and +0 for field 0 (whatever its sign and mantissa bits).
+ *   codes   device, lgn_codes_bytes(n, fmt->nbits) bytes, 16-byte aligned, read only
+ *   fmt     host; the format the stream was written with
+ *   out_dt  type of the output tensor (need not be the type that was quantised)
+ *   out     device, n elements of out_dt, 32-byte aligned, must not overlap codes
+ * Every value of a format has at most 7 significant bits, so the result is exact in
+ * both output types as long as the format's exponents are normal fp32 exponents:
+ * a format with 127 + scale_exp - E_max < 0 or scale_exp + E_max > 128 returns
+ * LGN_ERR_UNSUPPORTED (nothing is enqueued).  One launch, no workspace. */
+lgn_status lgn_dequantize(const void *codes, uint64_t n, const lgn_fp_format_t *fmt, lgn_dtype out_dt,
+                          void *out, void *stream);
+
 /* Self-test of the bounded device-side wait (no counterpart in the paper).
  * Same arguments and the same work as lgn_compress_layers, except that one
  * statistics tile of layer 0 is withheld from the queue, so layer 0's closed form

@@ -90,6 +90,8 @@ _lib.lgn_prefix_encode.argtypes = [_vp, _u64, _i32, C.c_double, _u64, _i32, _vp,
 _lib.lgn_prefix_encode.restype = _i32
 _lib.lgn_prefix_decode.argtypes = [_vp, _vp, _u64, _i32, C.c_double, _vp, _vp, _vp]
 _lib.lgn_prefix_decode.restype = _i32
+_lib.lgn_dequantize.argtypes = [_vp, _u64, C.POINTER(FpFormatT), _i32, _vp, _vp]
+_lib.lgn_dequantize.restype = _i32
 _lib.lgn_launches_per_call.argtypes = [_i32]
 _lib.lgn_launches_per_call.restype = _i32
 _lib.lgn_stats_static_scratch.argtypes = [_vp, _u64, _i32, _vp, _vp]
@@ -220,6 +222,18 @@ def lgn_quantize(g: torch.Tensor, fmt: Dict[str, int], rounding: int, seed: int,
     f = _fmt_struct(fmt)
     _check(_lib.lgn_quantize(_dev(g, "g"), _dev(out, "codes"), g.numel(), dtype_code(g), C.byref(f),
                              int(rounding), int(seed), _stream(stream)), "lgn_quantize")
+    return out
+
+
+def lgn_dequantize(codes: torch.Tensor, n: int, fmt: Dict[str, int], out: torch.Tensor, stream=None) -> torch.Tensor:
+    """Decode ``n`` packed codes (uint8 CUDA tensor) into ``out`` (float32 or bfloat16, n elements)."""
+    if out.numel() != n:
+        raise ValueError("out must hold n elements")
+    if codes.numel() * codes.element_size() < lgn_codes_bytes(n, fmt["nbits"]):
+        raise ValueError("codes shorter than lgn_codes_bytes(n, nbits)")
+    f = _fmt_struct(fmt)
+    _check(_lib.lgn_dequantize(_dev(codes, "codes") if n else None, n, C.byref(f), dtype_code(out),
+                               _dev(out, "out") if n else None, _stream(stream)), "lgn_dequantize")
     return out
 
 

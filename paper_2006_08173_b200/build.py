@@ -9,7 +9,8 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "liblgn.so")
-SOURCES = [os.path.join(_CSRC, "lgn.cu"), os.path.join(_CSRC, "lgn_prefix.cu")]
+SOURCES = [os.path.join(_CSRC, "lgn.cu"), os.path.join(_CSRC, "lgn_prefix.cu"),
+           os.path.join(_CSRC, "lgn_dequant.cu")]
 _DEPS = SOURCES + [os.path.join(_CSRC, "lgn_device.cuh"), os.path.join(_CSRC, "lgn_closed_form.cuh"),
                    os.path.join(_ROOT, "include", "lgn.h")]
 

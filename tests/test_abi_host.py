@@ -153,3 +153,23 @@ def test_device_entry_points_reject_bad_arguments_before_any_cuda_call(lgn):
     assert call(layer(), res=None) == INVALID
     assert call(layer(), n=-1) == INVALID
     assert call(layer(), n=0) == 0
+
+
+def test_dequantize_rejects_bad_arguments_before_any_cuda_call(lgn):
+    R = lgn.raw()
+    A, B = 0x10000, 0x90000
+    INVALID, UNSUPPORTED = 1, 2
+    ok = lgn.FpFormatT(6, 4, 1, -17)
+    assert R.lgn_dequantize(A, 100, None, 0, B, None) == INVALID
+    assert R.lgn_dequantize(A, 100, C.byref(lgn.FpFormatT(3, 1, 1, 0)), 0, B, None) == UNSUPPORTED
+    assert R.lgn_dequantize(A, 100, C.byref(lgn.FpFormatT(6, 4, 2, 0)), 0, B, None) == INVALID
+    assert R.lgn_dequantize(A, 100, C.byref(ok), 2, B, None) == INVALID                              # output type
+    assert R.lgn_dequantize(A, 100, C.byref(lgn.FpFormatT(6, 4, 1, -120)), 0, B, None) == UNSUPPORTED  # subnormal codes
+    assert R.lgn_dequantize(A, 100, C.byref(lgn.FpFormatT(6, 4, 1, 121)), 0, B, None) == UNSUPPORTED   # codes beyond fp32
+    assert R.lgn_dequantize(None, 100, C.byref(ok), 0, B, None) == INVALID
+    assert R.lgn_dequantize(A, 100, C.byref(ok), 0, None, None) == INVALID
+    assert R.lgn_dequantize(A, 100, C.byref(ok), 0, B + 16, None) == INVALID                         # out: 32-byte aligned
+    assert R.lgn_dequantize(A + 4, 100, C.byref(ok), 0, B, None) == INVALID
+    assert R.lgn_dequantize(A, 100, C.byref(ok), 0, A + 64, None) == INVALID                         # overlap
+    assert R.lgn_dequantize(A, 2 ** 50, C.byref(ok), 0, B, None) == UNSUPPORTED
+    assert R.lgn_dequantize(None, 0, C.byref(ok), 0, None, None) == 0                                # empty
