@@ -47,6 +47,12 @@ def _L():
         u32, u64, i32, dbl, vp = C.c_uint32, C.c_uint64, C.c_int, C.c_double, C.c_void_p
         lib.orc_stats.argtypes = [vp, u64, i32, C.POINTER(_Stats)]
         lib.orc_stats.restype = None
+        lib.orc_stats_masked.argtypes = [vp, vp, u64, i32, C.POINTER(_Stats), C.POINTER(u64)]
+        lib.orc_stats_masked.restype = None
+        lib.orc_max_abs.argtypes = [vp, u64, i32]
+        lib.orc_max_abs.restype = dbl
+        lib.orc_scale_exp_from_max.argtypes = [dbl, i32]
+        lib.orc_scale_exp_from_max.restype = i32
         lib.orc_philox4x32.argtypes = [vp, vp, i32, vp]
         lib.orc_philox4x32.restype = None
         lib.orc_rand16.argtypes = [u64, u64]
@@ -124,6 +130,37 @@ def stats(g: np.ndarray) -> dict:
     st = _Stats()
     _L().orc_stats(_ptr(g), g.size, _dtype_of(g), C.byref(st))
     return {"n": st.n, "nnz": st.nnz, "mu": st.mu, "sigma": st.sigma, "zero_frac": st.zero_frac}
+
+
+def stats_masked(g: np.ndarray, right_mode: np.ndarray) -> dict:
+    """Appendix A.9 steps (1), (3): l from the mask, mu and sigma over the right mode
+    (right_mode[i] != 0).  ``n_right`` = size of the right mode."""
+    g = _flat(g)
+    m = np.ascontiguousarray(right_mode, dtype=np.uint8).reshape(-1)
+    assert m.size == g.size
+    st = _Stats()
+    nr = C.c_uint64()
+    _L().orc_stats_masked(_ptr(g), _ptr(m), g.size, _dtype_of(g), C.byref(st), C.byref(nr))
+    return {"n": st.n, "nnz": st.nnz, "mu": st.mu, "sigma": st.sigma, "zero_frac": st.zero_frac,
+            "n_right": nr.value}
+
+
+def max_abs(g: np.ndarray) -> float:
+    g = _flat(g)
+    return float(_L().orc_max_abs(_ptr(g), g.size, _dtype_of(g)))
+
+
+def scale_exp_from_max(max_abs_: float, exp_bits: int) -> int:
+    """Algorithm 1's scale read as: the largest element lands in the top binade."""
+    return int(_L().orc_scale_exp_from_max(max_abs_, exp_bits))
+
+
+def fp_format_max_scale(mu: float, sigma: float, nnz: int, nbits: int, max_abs_: float) -> dict:
+    """Split from Eq. 4 as in fp_format; scale from the tensor's maximum."""
+    f = fp_format(mu, sigma, nnz, nbits)
+    if nnz:
+        f["scale_exp"] = scale_exp_from_max(max_abs_, f["exp_bits"])
+    return f
 
 
 # --------------------------------------------------------------------------- rng

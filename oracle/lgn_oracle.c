@@ -24,6 +24,14 @@
  *                      derivation of Eq. 4; Monte-Carlo with orc_quantize
  *   orc_quantize_*     brute force over every code of every format
  *   orc_philox4x32     known-answer vectors published with the generator (10 rounds)
+ *   orc_stats_masked   hand cases (powers of two under a hand-written mask); recovery of the
+ *                      right mode's generator parameters and of l on a two-mode tensor;
+ *                      the identity l + (1-l) S' = S as achieved sparsity when the left mode
+ *                      lies orders of magnitude below the right one (Appendix A.9)
+ *   orc_scale_exp_from_max
+ *                      powers of two and their neighbours by hand; the largest element's
+ *                      exponent lands on E_max - 1 (checked with frexp in the test); no
+ *                      element is clipped before rounding
  *   orc_dequantize     every code of every format against the value formula of Eq. 1-2
  *                      written out in the test; quantising the decoded value (nearest)
  *                      gives the code back
@@ -121,6 +129,79 @@ void orc_stats(const void *g, uint64_t n, int dtype, orc_stats_t *out)
     out->mu = mu;
     out->sigma = nnz ? sqrt(ss / (double)nnz) : 0.0;
     out->zero_frac = n ? 1.0 - (double)nnz / (double)n : 0.0;
+}
+
+/* Appendix "bi-modal lognormal pruning", steps (1) and (3).  The gradient before
+ * batch-norm has two modes; they are told apart by the SAME entry of the gradient
+ * after batch-norm (after the ReLU's backward): zero there -> left mode, non-zero
+ * -> right mode.  right_mode[i] != 0 marks the right-mode entries (one byte each).
+ *   l         = (entries of the left mode) / n                      step (1)
+ *   mu, sigma = mean and std of ln|g| over the right-mode entries   step (3)
+ * (a right-mode entry that is itself exactly zero has no logarithm and is left
+ * out of the mean and the deviation, like in orc_stats; it still counts as
+ * right mode in l).  out->nnz is the number of entries that entered mu and sigma;
+ * out->zero_frac is l.  *n_right receives the size of the right mode. */
+void orc_stats_masked(const void *g, const uint8_t *right_mode, uint64_t n, int dtype,
+                      orc_stats_t *out, uint64_t *n_right)
+{
+    uint64_t cnt = 0, right = 0;
+    double sum = 0.0, comp = 0.0;
+    for (uint64_t i = 0; i < n; ++i) {
+        if (!right_mode[i]) continue;
+        ++right;
+        double x = elem(g, dtype, i);
+        if (x == 0.0) continue;
+        double y = log(fabs(x)) - comp;
+        double t = sum + y;
+        comp = (t - sum) - y;
+        sum = t;
+        ++cnt;
+    }
+    double mu = cnt ? sum / (double)cnt : 0.0;
+    double ss = 0.0; comp = 0.0;
+    for (uint64_t i = 0; i < n; ++i) {
+        if (!right_mode[i]) continue;
+        double x = elem(g, dtype, i);
+        if (x == 0.0) continue;
+        double d = log(fabs(x)) - mu;
+        double y = d * d - comp;
+        double t = ss + y;
+        comp = (t - ss) - y;
+        ss = t;
+    }
+    out->n = n;
+    out->nnz = cnt;
+    out->mu = mu;
+    out->sigma = cnt ? sqrt(ss / (double)cnt) : 0.0;
+    out->zero_frac = n ? 1.0 - (double)right / (double)n : 0.0;
+    *n_right = right;
+}
+
+/* max |g| over the whole tensor (Algorithm 1, "max(|X|)"). */
+double orc_max_abs(const void *g, uint64_t n, int dtype)
+{
+    double m = 0.0;
+    for (uint64_t i = 0; i < n; ++i) {
+        double a = fabs(elem(g, dtype, i));
+        if (a > m) m = a;
+    }
+    return m;
+}
+
+/* Algorithm 1, the scale from the maximum.  The printed line
+ * "mu_l = floor(log2 max|X|) / log2(E_max)" does not give an exponent shift as it
+ * stands; the text around it fixes what it is for: the scale "sacrifices the
+ * smallest elements to keep the largest gradients magnitude representable".  With
+ * representable exponents -E_max+1 .. E_max-1 that is the power of two that puts
+ * the largest element in the top binade:
+ *     e_s = floor(log2 max|X|) - (E_max - 1).
+ * max_abs must be > 0. */
+int orc_scale_exp_from_max(double max_abs, int n2)
+{
+    int ex;
+    (void)frexp(max_abs, &ex);            /* max_abs = f * 2^ex, f in [0.5, 1): floor(log2) = ex - 1 */
+    int Emax = 1 << (n2 - 1);
+    return (ex - 1) - (Emax - 1);
 }
 
 /* ------------------------------------------------------------------ */

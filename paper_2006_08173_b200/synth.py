@@ -57,6 +57,29 @@ def lognormal_tensor(n: int, mu: float, sigma: float, zero_frac: float, seed: in
     return out
 
 
+def bimodal_tensor(n: int, mu_right: float, sigma_right: float, mu_left: float, sigma_left: float,
+                   left_frac: float, seed: int, dtype: torch.dtype = torch.float32, device: str = "cpu"):
+    """A gradient before batch-norm and the mask that tells its two modes apart
+    (the entries where the gradient after batch-norm is non-zero): returns
+    (g, right_mode).  right_mode is a uint8 tensor, 1 with probability
+    1 - left_frac; g is dense, sign * exp(N(mu_right, sigma_right^2)) where the
+    mask is 1 and sign * exp(N(mu_left, sigma_left^2)) elsewhere."""
+    gen = torch.Generator(device=device)
+    gen.manual_seed(int(seed))
+    g = torch.empty(n, dtype=dtype, device=device)
+    mask = torch.empty(n, dtype=torch.uint8, device=device)
+    for lo in range(0, n, _CHUNK):
+        m = min(_CHUNK, n - lo)
+        z = torch.randn(m, generator=gen, device=device, dtype=torch.float64)
+        u_sign = torch.rand(m, generator=gen, device=device)
+        right = torch.rand(m, generator=gen, device=device) >= left_frac
+        y = torch.where(right, mu_right + sigma_right * z, mu_left + sigma_left * z)
+        mag = torch.exp(y)
+        g[lo:lo + m] = torch.where(u_sign < 0.5, -mag, mag).to(torch.float32).to(dtype)
+        mask[lo:lo + m] = right.to(torch.uint8)
+    return g, mask
+
+
 def as_numpy_bits(t: torch.Tensor) -> np.ndarray:
     """Host numpy view of a tensor: float32 stays float32, bfloat16 becomes its
     raw uint16 bit patterns (numpy has no bfloat16)."""
