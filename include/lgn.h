@@ -53,6 +53,14 @@ typedef enum {
 typedef enum { LGN_F32 = 0, LGN_BF16 = 1 } lgn_dtype;
 typedef enum { LGN_ROUND_NEAREST = 0, LGN_ROUND_STOCHASTIC = 1 } lgn_rounding;
 typedef enum { LGN_MODE_PRUNE = 0, LGN_MODE_QUANTIZE = 1 } lgn_mode;
+/* Where a quantised layer's power-of-two scale comes from (Algorithm 1):
+ *   LGN_SCALE_CENTRED   e_s = floor(mu/ln 2 + 1/2): the median magnitude sits in the middle
+ *                       of the format's range, the setting Eq. 4 is derived for
+ *   LGN_SCALE_FROM_MAX  e_s = floor(log2 max|g|) - (E_max - 1): the largest element sits in
+ *                       the top binade, nothing is clipped, the smallest elements are given
+ *                       up ("sacrifices the smallest elements to keep the largest gradients
+ *                       magnitude representable", appendix "Gradient scaling") */
+typedef enum { LGN_SCALE_CENTRED = 0, LGN_SCALE_FROM_MAX = 1 } lgn_scale_mode;
 
 /* Lognormal statistics of one tensor (Section 3: magnitudes, zeros left out). */
 typedef struct {
@@ -127,6 +135,11 @@ double lgn_snap_threshold(double tau, lgn_dtype dt);
  *   fmt  host, receives the format.  sigma is clamped to [1e-6, 25]. */
 lgn_status lgn_fp_format(double mu, double sigma, int nbits, lgn_fp_format_t *fmt);
 
+/* Algorithm 1's scale taken from the tensor's maximum, for a format with exp_bits
+ * exponent bits: e_s = floor(log2 max_abs) - (2^(exp_bits-1) - 1).  Host only.
+ * max_abs must be finite and > 0, exp_bits in 1..7. */
+lgn_status lgn_scale_from_max(double max_abs, int exp_bits, int32_t *scale_exp);
+
 /* Stochastic pruning with a given threshold (Eq. 5): the steady-state call
  * between refreshes of the statistics.
  *   g, out  device, n elements of dt; out has the same type and layout
@@ -170,17 +183,29 @@ typedef struct {
     int32_t      rounding;   /* quantize: lgn_rounding                                     */
     uint64_t     seed;
     int32_t      use_override;   /* nonzero: use mu_override/sigma_override in the closed  */
-    int32_t      reserved;       /* form instead of the measured mu/sigma (nnz and the     */
+    int32_t      scale_mode;     /* form instead of the measured mu/sigma (nnz and the     */
     double       mu_override;    /* zero fraction are always the measured ones)            */
-    double       sigma_override;
+    double       sigma_override; /* scale_mode: quantize only, lgn_scale_mode; 0 for prune  */
+    /* Bi-modal pruning (appendix "Algorithm for bi-modal lognormal pruning"), prune only,
+     * NULL otherwise.  Device, n bytes, 16-byte aligned: byte i != 0 says that entry i
+     * belongs to the RIGHT mode, i.e. that the same entry of the gradient after
+     * batch-norm (the one the ReLU's backward produced) is non-zero; g itself is the
+     * dense gradient before batch-norm.  With a mask, l is the fraction of left-mode
+     * entries (step 1), mu and sigma are taken over the right-mode entries of g only
+     * (step 3), S' = (S - l)/(1 - l) (step 2), and the threshold so obtained prunes the
+     * WHOLE tensor (step 4). */
+    const void  *right_mode;
 } lgn_layer_t;
 
 typedef struct {
-    lgn_stats_t      stats;   /* measured, whatever the override says                     */
+    lgn_stats_t      stats;   /* measured, whatever the override says; with a right_mode   */
+                              /* mask: nnz, sums, mu, sigma are over the right mode only    */
     double           tau;     /* prune: the threshold used (already snapped); else 0       */
     lgn_fp_format_t  fmt;     /* quantize: the format used; else zeros                     */
     int32_t          status;  /* lgn_status of this layer (LGN_ERR_TIMEOUT: output invalid) */
-    int32_t          reserved;
+    float            max_abs; /* max|g| over the whole tensor; measured only for layers     */
+                              /* with LGN_SCALE_FROM_MAX or a right_mode mask, else 0       */
+    uint64_t         n_right_mode;  /* with a mask: entries whose mask byte != 0; else 0   */
 } lgn_layer_result_t;
 
 /* The whole path for a list of tensors in one kernel launch (plus one tiny
@@ -224,7 +249,11 @@ lgn_status lgn_compress_layers(const lgn_layer_t *layers, int num_layers,
  * capacity that always suffices.  ws: device scratch of
  * lgn_prefix_workspace_bytes(n) bytes, 16-byte aligned, free again when the call's
  * work on `stream` has finished.  Errors: as for the other entry points; n above
- * 2^34 is LGN_ERR_UNSUPPORTED.  Three launches, no allocation, no synchronisation.
+ * 2^34 is LGN_ERR_UNSUPPORTED.  One memset of the workspace and one launch, no
+ * allocation, no synchronisation.  Blocks obtain their first word from the lengths the
+ * blocks before them have published; these device-side waits are bounded, and if one
+ * runs out (it cannot while the GPU makes progress) off_dev[nblocks] is set to
+ * 2^64 - 1, which the caller sees as "does not fit".
  * lgn_prefix_decode is the inverse: n elements of type dt into out_dev. */
 #define LGN_PREFIX_BLOCK 2048u
 uint64_t   lgn_prefix_blocks(uint64_t n);

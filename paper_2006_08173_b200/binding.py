@@ -26,6 +26,7 @@ LGN_OK = 0
 F32, BF16 = 0, 1
 ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
 MODE_PRUNE, MODE_QUANTIZE = 0, 1
+SCALE_CENTRED, SCALE_FROM_MAX = 0, 1
 
 
 class StatsT(C.Structure):
@@ -42,16 +43,16 @@ class LayerT(C.Structure):
     _fields_ = [("g", C.c_void_p), ("out", C.c_void_p), ("n", C.c_uint64),
                 ("dt", C.c_int32), ("mode", C.c_int32), ("S", C.c_double),
                 ("nbits", C.c_int32), ("rounding", C.c_int32), ("seed", C.c_uint64),
-                ("use_override", C.c_int32), ("reserved", C.c_int32),
-                ("mu_override", C.c_double), ("sigma_override", C.c_double)]
+                ("use_override", C.c_int32), ("scale_mode", C.c_int32),
+                ("mu_override", C.c_double), ("sigma_override", C.c_double), ("right_mode", C.c_void_p)]
 
 
 class LayerResultT(C.Structure):
     _fields_ = [("stats", StatsT), ("tau", C.c_double), ("fmt", FpFormatT),
-                ("status", C.c_int32), ("reserved", C.c_int32)]
+                ("status", C.c_int32), ("max_abs", C.c_float), ("n_right_mode", C.c_uint64)]
 
 
-assert C.sizeof(StatsT) == 48 and C.sizeof(LayerT) == 80 and C.sizeof(LayerResultT) == 80
+assert C.sizeof(StatsT) == 48 and C.sizeof(LayerT) == 88 and C.sizeof(LayerResultT) == 88
 
 _vp, _u64, _sz, _dbl, _i32 = C.c_void_p, C.c_uint64, C.c_size_t, C.c_double, C.c_int
 _lib.lgn_status_string.argtypes = [_i32]
@@ -68,6 +69,8 @@ _lib.lgn_snap_threshold.argtypes = [_dbl, _i32]
 _lib.lgn_snap_threshold.restype = _dbl
 _lib.lgn_fp_format.argtypes = [_dbl, _dbl, _i32, C.POINTER(FpFormatT)]
 _lib.lgn_fp_format.restype = _i32
+_lib.lgn_scale_from_max.argtypes = [_dbl, _i32, C.POINTER(C.c_int32)]
+_lib.lgn_scale_from_max.restype = _i32
 _lib.lgn_prune.argtypes = [_vp, _vp, _u64, _i32, _dbl, _u64, _vp]
 _lib.lgn_prune.restype = _i32
 _lib.lgn_quantize.argtypes = [_vp, _vp, _u64, _i32, C.POINTER(FpFormatT), _i32, _u64, _vp]
@@ -172,6 +175,12 @@ def lgn_fp_format(mu: float, sigma: float, nbits: int) -> Dict[str, int]:
     return {"nbits": f.nbits, "exp_bits": f.exp_bits, "man_bits": f.man_bits, "scale_exp": f.scale_exp}
 
 
+def lgn_scale_from_max(max_abs: float, exp_bits: int) -> int:
+    e = C.c_int32()
+    _check(_lib.lgn_scale_from_max(float(max_abs), int(exp_bits), C.byref(e)), "lgn_scale_from_max")
+    return e.value
+
+
 def _fmt_struct(fmt: Dict[str, int]) -> FpFormatT:
     return FpFormatT(fmt["nbits"], fmt["exp_bits"], fmt["man_bits"], fmt["scale_exp"])
 
@@ -239,18 +248,25 @@ def lgn_dequantize(codes: torch.Tensor, n: int, fmt: Dict[str, int], out: torch.
 
 def make_layer(g: torch.Tensor, out: torch.Tensor, mode: int, S: float = 0.0, nbits: int = 0,
                rounding: int = ROUND_NEAREST, seed: int = 0, mu_override: Optional[float] = None,
-               sigma_override: Optional[float] = None) -> LayerT:
+               sigma_override: Optional[float] = None, scale_mode: int = SCALE_CENTRED,
+               right_mode: Optional[torch.Tensor] = None) -> LayerT:
+    """``right_mode``: uint8/bool CUDA tensor of g.numel() bytes (bi-modal pruning), or None."""
     use = mu_override is not None and sigma_override is not None
+    mask = None
+    if right_mode is not None:
+        if right_mode.element_size() != 1 or right_mode.numel() != g.numel():
+            raise ValueError("right_mode must hold one byte per element of g")
+        mask = _dev(right_mode, "right_mode") if g.numel() else None
     return LayerT(_dev(g, "g") if g.numel() else (g.data_ptr() or None),
                   _dev(out, "out") if out.numel() else (out.data_ptr() or None), g.numel(), dtype_code(g),
-                  mode, float(S), int(nbits), int(rounding), int(seed), 1 if use else 0, 0,
-                  float(mu_override) if use else 0.0, float(sigma_override) if use else 0.0)
+                  mode, float(S), int(nbits), int(rounding), int(seed), 1 if use else 0, int(scale_mode),
+                  float(mu_override) if use else 0.0, float(sigma_override) if use else 0.0, mask)
 
 
 def lgn_compress_layers(layers: Sequence[LayerT], results_dev: torch.Tensor, ws: torch.Tensor,
                         stream=None) -> None:
     """Enqueue the grouped path.  ``results_dev``: uint8 CUDA tensor of at least
-    80 bytes per layer; ``ws``: uint8 CUDA tensor of lgn_workspace_bytes(...)."""
+    88 bytes per layer; ``ws``: uint8 CUDA tensor of lgn_workspace_bytes(...)."""
     L = len(layers)
     arr = (LayerT * max(1, L))(*layers)
     if results_dev.numel() * results_dev.element_size() < L * C.sizeof(LayerResultT):
@@ -284,7 +300,7 @@ def read_results(results_dev: torch.Tensor, num_layers: int) -> List[Dict]:
                     "mu": r.stats.mu, "sigma": r.stats.sigma, "tau": r.tau,
                     "fmt": {"nbits": r.fmt.nbits, "exp_bits": r.fmt.exp_bits, "man_bits": r.fmt.man_bits,
                             "scale_exp": r.fmt.scale_exp},
-                    "status": r.status})
+                    "status": r.status, "max_abs": r.max_abs, "n_right_mode": r.n_right_mode})
     return out
 
 
@@ -294,7 +310,7 @@ def _result_dict(r: LayerResultT) -> Dict:
             "mu": r.stats.mu, "sigma": r.stats.sigma, "tau": r.tau,
             "fmt": {"nbits": r.fmt.nbits, "exp_bits": r.fmt.exp_bits, "man_bits": r.fmt.man_bits,
                     "scale_exp": r.fmt.scale_exp},
-            "status": r.status}
+            "status": r.status, "max_abs": r.max_abs, "n_right_mode": r.n_right_mode}
 
 
 def make_host_layer(g: torch.Tensor, out: torch.Tensor, mode: int, **kw) -> LayerT:
@@ -303,7 +319,8 @@ def make_host_layer(g: torch.Tensor, out: torch.Tensor, mode: int, **kw) -> Laye
         raise ValueError("host layers take contiguous CPU tensors")
     lay = LayerT(g.data_ptr() or None, out.data_ptr() or None, g.numel(), dtype_code(g), mode,
                  float(kw.get("S", 0.0)), int(kw.get("nbits", 0)), int(kw.get("rounding", ROUND_NEAREST)),
-                 int(kw.get("seed", 0)), 0, 0, 0.0, 0.0)
+                 int(kw.get("seed", 0)), 0, int(kw.get("scale_mode", SCALE_CENTRED)), 0.0, 0.0,
+                 (kw["right_mode"].data_ptr() or None) if kw.get("right_mode") is not None else None)
     return lay
 
 

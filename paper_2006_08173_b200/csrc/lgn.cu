@@ -48,9 +48,18 @@ struct alignas(16) LayerState {          // written by the set-up launch, then r
     lgn_layer_result_t *result_out;      // may be null
     uint32_t            ntiles;
     uint32_t            partial0;        // first slot of this layer in the partial array
-    int32_t             dt, mode, nbits, rounding, use_override, pad;
+    int32_t             dt, mode, nbits, rounding, use_override, scale_mode;
+    const uint8_t      *mask;            // right-mode mask of a bi-modal gradient, or null
+    uint64_t            pad;
 };
-static_assert(sizeof(LayerState) == 112, "LayerState layout");
+static_assert(sizeof(LayerState) == 128, "LayerState layout");
+
+// Layers that need the extended statistics tile (mask and / or max|g|); their
+// statistics runs carry phase kPhaseStatsExt in the queue.
+static inline bool needs_ext_stats(const LayerState &L) {
+    return L.mask != nullptr || L.scale_mode == LGN_SCALE_FROM_MAX;
+}
+constexpr uint32_t kPhaseStats = 0, kPhaseApply = 1, kPhaseStatsExt = 2;
 
 struct alignas(16) LayerDyn {            // zeroed by the set-up launch, written by the kernel
     uint32_t    done;                    // statistics tiles completed
@@ -65,7 +74,7 @@ struct alignas(16) Segment {             // a run of consecutive queue items
     uint32_t first_item;
     uint32_t ntiles;
     uint32_t layer;
-    uint32_t phase;                      // 0 statistics, 1 apply
+    uint32_t phase;                      // 0 statistics, 1 apply, 2 statistics with a mask and / or max|g|
     uint32_t tile_begin;                 // first tile of the layer this run covers
     uint32_t reverse;                    // walk the run from its last tile down
     uint32_t pad[2];
@@ -75,8 +84,10 @@ static_assert(sizeof(Segment) == 32, "Segment layout");
 struct alignas(16) Partial {
     double             s1, s2;           // sums of log2|g| and its square over the tile's nonzeros
     unsigned long long cnt;
-    unsigned long long pad;
+    uint32_t           right;            // extended tiles: entries of the right mode in the tile; else 0
+    float              amax;             // extended tiles: largest magnitude in the tile; else 0
 };
+static_assert(sizeof(Partial) == 32, "Partial layout");
 
 struct WsLayout {
     size_t states, dyn, segs, partials, total;
@@ -136,20 +147,21 @@ __device__ __forceinline__ void st_release(uint32_t *p, uint32_t v) {
 // specialised kernels inline, and one general body (ragged last tile, any layer
 // scale, any threshold) kept out of line so that it costs the hot path no
 // registers.
+// The out-of-line statistics tile: ragged last tiles, and the extended form (a
+// right-mode mask and / or max|g|).  Does the whole item: the tile, the CTA
+// reduction (one barrier) and the partial.
 template <int DT>
-__device__ __noinline__ void stats_tile_general(const void *g, uint64_t base, uint64_t n, StatsAcc &acc) {
-    stats_tile<DT, false>(g, base, n, acc);
-}
+__device__ __noinline__ void run_stats_tile_slow(const LayerState &L, uint32_t tile, bool ext, Partial *partials, double *sm);
 
 // One tile's sums: per-warp shuffle tree, eight warp results through shared
 // memory, added in warp order by thread 0, which also stores the tile's partial.
 // One barrier; `sm` is reused only after the caller's next barrier.
 template <int DT, bool INLINE_HOT>
-__device__ __forceinline__ void run_stats_tile(const LayerState &L, uint32_t tile, Partial *partials, double *sm) {
-    StatsAcc acc;
+__device__ __forceinline__ void run_stats_tile(const LayerState &L, uint32_t tile, bool ext, Partial *partials, double *sm) {
     const uint64_t base = (uint64_t)tile * kTileElems;
-    if (INLINE_HOT && base + kTileElems <= L.n) stats_tile<DT, true>(L.g, base, L.n, acc);
-    else                                        stats_tile_general<DT>(L.g, base, L.n, acc);
+    if (!INLINE_HOT || ext || base + kTileElems > L.n) { run_stats_tile_slow<DT>(L, tile, ext, partials, sm); return; }
+    StatsAcc acc;
+    stats_tile<DT, true>(L.g, base, L.n, acc);
     #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
         acc.s1 += __shfl_down_sync(0xFFFFFFFFu, acc.s1, off);
@@ -163,11 +175,39 @@ __device__ __forceinline__ void run_stats_tile(const LayerState &L, uint32_t til
     __syncthreads();
     if (threadIdx.x == 0) {
         Partial p;
-        p.s1 = 0.0; p.s2 = 0.0; p.cnt = 0; p.pad = 0;
+        p.s1 = 0.0; p.s2 = 0.0; p.cnt = 0; p.right = 0u; p.amax = 0.f;
         #pragma unroll
         for (int k = 0; k < kWarps; ++k) {
             p.s1 += sm[k]; p.s2 += sm[kWarps + k];
             p.cnt += (unsigned long long)__double_as_longlong(sm[2 * kWarps + k]);
+        }
+        partials[L.partial0 + tile] = p;
+    }
+}
+
+template <int DT>
+__device__ __noinline__ void run_stats_tile_slow(const LayerState &L, uint32_t tile, bool ext, Partial *partials, double *sm) {
+    StatsAcc acc;
+    const uint64_t base = (uint64_t)tile * kTileElems;
+    if (!ext)        stats_tile<DT, false>(L.g, base, L.n, acc);
+    else if (L.mask) stats_tile_ext<DT, true>(L.g, L.mask, base, L.n, acc);
+    else             stats_tile_ext<DT, false>(L.g, nullptr, base, L.n, acc);
+    warp_reduce(acc, 32);
+    const int w = threadIdx.x >> 5;
+    if ((threadIdx.x & 31) == 0) {
+        sm[w] = acc.s1; sm[kWarps + w] = acc.s2; sm[2 * kWarps + w] = __longlong_as_double((long long)acc.cnt);
+        sm[3 * kWarps + w] = __longlong_as_double((long long)acc.right); sm[4 * kWarps + w] = (double)acc.amax;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        Partial p;
+        p.s1 = 0.0; p.s2 = 0.0; p.cnt = 0; p.right = 0u; p.amax = 0.f;
+        #pragma unroll
+        for (int k = 0; k < kWarps; ++k) {
+            p.s1 += sm[k]; p.s2 += sm[kWarps + k];
+            p.cnt += (unsigned long long)__double_as_longlong(sm[2 * kWarps + k]);
+            p.right += (uint32_t)__double_as_longlong(sm[3 * kWarps + k]);
+            p.amax = fmaxf(p.amax, (float)sm[4 * kWarps + k]);
         }
         partials[L.partial0 + tile] = p;
     }
@@ -224,6 +264,18 @@ __device__ __forceinline__ void run_quant_tile_any(const void *g, void *out, uin
     #undef LGN_Q
 }
 
+// floor(log2 a) of a positive finite fp32 value, from its pattern (subnormals included).
+__host__ __device__ inline int floor_log2_f32(float a) {
+    uint32_t b;
+    memcpy(&b, &a, 4);
+    b &= 0x7FFFFFFFu;
+    const int e = (int)(b >> 23);
+    if (e) return e - 127;
+    int top = -1;
+    for (int k = 22; k >= 0; --k) if ((b >> k) & 1u) { top = k; break; }
+    return top - 149;
+}
+
 // Adds up a layer's partials (thread t takes slots t, t+kThreads, ... in order,
 // then the fixed tree), turns them into mu, sigma, and evaluates the closed form.
 __device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn *D, const Partial *partials, double *sm) {
@@ -233,6 +285,8 @@ __device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn *D, co
         acc.s1 += __ldcg(&p->s1);
         acc.s2 += __ldcg(&p->s2);
         acc.cnt += __ldcg(&p->cnt);
+        acc.right += __ldcg(&p->right);
+        acc.amax = fmaxf(acc.amax, __ldcg(&p->amax));
     }
     block_reduce(acc, sm);
     if (threadIdx.x != 0) return;
@@ -259,7 +313,8 @@ __device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn *D, co
     lgn_fp_format_t fmt;
     fmt.nbits = fmt.exp_bits = fmt.man_bits = fmt.scale_exp = 0;
     if (L.mode == LGN_MODE_PRUNE) {
-        const double zero_frac = 1.0 - (double)st.nnz / (double)st.n;
+        // l: the exact zeros, or with a mask the left mode (appendix, bi-modal pruning, step 1)
+        const double zero_frac = 1.0 - (double)(L.mask ? acc.right : st.nnz) / (double)st.n;
         const double tau = acc.cnt ? threshold_for(mu, sigma, zero_frac, L.S) : 0.0;
         const float t = (L.dt == LGN_BF16) ? snap_threshold_bf16(tau) : snap_threshold_f32(tau);
         D->tau = t;
@@ -267,6 +322,8 @@ __device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn *D, co
     } else if (L.mode == LGN_MODE_QUANTIZE) {
         if (acc.cnt) {
             choose_format(mu, sigma, L.nbits, fmt);
+            if (L.scale_mode == LGN_SCALE_FROM_MAX)               // Algorithm 1: the maximum in the top binade
+                fmt.scale_exp = floor_log2_f32(acc.amax) - ((1 << (fmt.exp_bits - 1)) - 1);
         } else {                                              // all zero: every code is 0 anyway
             fmt.nbits = L.nbits; fmt.exp_bits = 1; fmt.man_bits = L.nbits - 2; fmt.scale_exp = 0;
         }
@@ -274,7 +331,8 @@ __device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn *D, co
     }
     if (L.result_out) {
         lgn_layer_result_t r;
-        r.stats = st; r.tau = tau_used; r.fmt = fmt; r.status = LGN_OK; r.reserved = 0;
+        r.stats = st; r.tau = tau_used; r.fmt = fmt; r.status = LGN_OK;
+        r.max_abs = acc.amax; r.n_right_mode = L.mask ? acc.right : 0ull;
         *L.result_out = r;
     }
     __threadfence();
@@ -301,7 +359,7 @@ template <int DT, int MODE, int NBITS, int SR>
 __global__ void __launch_bounds__(kThreads, kMinCtas)
 compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Segment *segs,
                 int num_layers, uint32_t total_items, Partial *partials) {
-    __shared__ double sm_red[3 * kWarps];
+    __shared__ double sm_red[5 * kWarps];
     __shared__ uint32_t sm_item[2];
     __shared__ uint32_t sm_fin[2];               // layer + 1 whose statistics this CTA has just completed
     __shared__ uint32_t sm_flag;
@@ -352,12 +410,13 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
         const LayerState &L = states[sg.layer];
         LayerDyn *D = dyn + sg.layer;
 
-        if (sg.phase == 0) {
+        if (sg.phase != kPhaseApply) {
+            const bool ext = sg.phase == kPhaseStatsExt;
             if constexpr (kSpecial) {
-                run_stats_tile<DT, true>(L, tile, partials, sm_red);
+                run_stats_tile<DT, true>(L, tile, ext, partials, sm_red);
             } else {
-                if (L.dt == LGN_BF16) run_stats_tile<LGN_BF16, false>(L, tile, partials, sm_red);
-                else                  run_stats_tile<LGN_F32, false>(L, tile, partials, sm_red);
+                if (L.dt == LGN_BF16) run_stats_tile<LGN_BF16, false>(L, tile, ext, partials, sm_red);
+                else                  run_stats_tile<LGN_F32, false>(L, tile, ext, partials, sm_red);
             }
             if (threadIdx.x == 0) {
                 __threadfence();                                   // the partial before the ticket
@@ -489,6 +548,19 @@ static lgn_status check_layer(const lgn_layer_t &d) {
         const char *a = static_cast<const char *>(d.g), *b = static_cast<const char *>(d.out);
         if (a < b + out_bytes && b < a + in_bytes) return LGN_ERR_INVALID_ARG;    // overlap
     }
+    if (d.mode == LGN_MODE_QUANTIZE) {
+        if (d.scale_mode != LGN_SCALE_CENTRED && d.scale_mode != LGN_SCALE_FROM_MAX) return LGN_ERR_INVALID_ARG;
+        if (d.right_mode != nullptr) return LGN_ERR_INVALID_ARG;       // the mask belongs to bi-modal pruning
+    } else {
+        if (d.scale_mode != 0) return LGN_ERR_INVALID_ARG;
+        if (d.right_mode != nullptr && d.mode != LGN_MODE_PRUNE) return LGN_ERR_INVALID_ARG;
+    }
+    if (d.right_mode != nullptr && d.n > 0) {
+        if (!aligned16(d.right_mode)) return LGN_ERR_INVALID_ARG;
+        const char *m = static_cast<const char *>(d.right_mode), *b = static_cast<const char *>(d.out);
+        const size_t out_bytes = d.n * (d.dt == LGN_BF16 ? 2u : 4u);
+        if (m < b + out_bytes && b < m + d.n) return LGN_ERR_INVALID_ARG;   // the output would overwrite the mask
+    }
     if (d.use_override && !(d.sigma_override >= 0.0 && std::isfinite(d.mu_override) && std::isfinite(d.sigma_override)))
         return LGN_ERR_INVALID_ARG;
     return LGN_OK;
@@ -514,7 +586,8 @@ static void build_queue(const std::vector<LayerState> &st, std::vector<Segment> 
         if (phase == 1 && st[layer].mode == kModeStatsOnly) return;
         Segment s;
         memset(&s, 0, sizeof s);
-        s.first_item = item; s.ntiles = st[layer].ntiles; s.layer = layer; s.phase = phase;
+        s.first_item = item; s.ntiles = st[layer].ntiles; s.layer = layer;
+        s.phase = phase == 1 ? kPhaseApply : (needs_ext_stats(st[layer]) ? kPhaseStatsExt : kPhaseStats);
         s.tile_begin = 0; s.reverse = phase;
         if (withhold_tile && layer == 0 && phase == 0) {   // self-test: layer 0 can never complete
             s.ntiles -= 1;
@@ -566,6 +639,8 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
         s.partial0 = partial0;
         s.dt = d.dt; s.mode = d.mode; s.nbits = d.nbits; s.rounding = d.rounding;
         s.use_override = d.use_override ? 1 : 0;
+        s.scale_mode = d.scale_mode;
+        s.mask = static_cast<const uint8_t *>(d.right_mode);
         partial0 += s.ntiles;
     }
     std::vector<Segment> segs;
@@ -691,6 +766,15 @@ extern "C" lgn_status lgn_fp_format(double mu, double sigma, int nbits, lgn_fp_f
     return LGN_OK;
 }
 
+extern "C" lgn_status lgn_scale_from_max(double max_abs, int exp_bits, int32_t *scale_exp) {
+    if (scale_exp == nullptr) return LGN_ERR_INVALID_ARG;
+    if (!(max_abs > 0.0) || !std::isfinite(max_abs) || exp_bits < 1 || exp_bits > 7) return LGN_ERR_INVALID_ARG;
+    int ex = 0;
+    (void)std::frexp(max_abs, &ex);                          // max_abs = f 2^ex, f in [1/2, 1)
+    *scale_exp = (ex - 1) - ((1 << (exp_bits - 1)) - 1);
+    return LGN_OK;
+}
+
 static int apply_grid(const void *fn, uint32_t ntiles) {
     int g = persistent_ctas(fn);
     if (g < 1) return -1;
@@ -768,14 +852,14 @@ extern "C" lgn_status lgn_compress_layers(const lgn_layer_t *layers, int num_lay
 // ------------------------------------------------------------------ host-buffer form
 namespace {
 struct StagingPlan {
-    std::vector<size_t> in_off, out_off, in_bytes, out_bytes;
+    std::vector<size_t> in_off, out_off, mask_off, in_bytes, out_bytes;
     size_t results_off = 0, ws_off = 0, ws_bytes = 0, total = 0;
 };
 
 bool plan_staging(const lgn_layer_t *layers, int L, StagingPlan &p) {
     size_t off = 0;
     std::vector<uint64_t> ns((size_t)L);
-    p.in_off.resize(L); p.out_off.resize(L); p.in_bytes.resize(L); p.out_bytes.resize(L);
+    p.in_off.resize(L); p.out_off.resize(L); p.mask_off.resize(L); p.in_bytes.resize(L); p.out_bytes.resize(L);
     for (int k = 0; k < L; ++k) {
         const lgn_layer_t &d = layers[k];
         if (d.dt != LGN_F32 && d.dt != LGN_BF16) return false;
@@ -786,6 +870,7 @@ bool plan_staging(const lgn_layer_t *layers, int L, StagingPlan &p) {
         p.out_bytes[k] = d.mode == LGN_MODE_PRUNE ? p.in_bytes[k] : lgn_codes_bytes(d.n, d.nbits);
         p.in_off[k] = off;  off += round_up(p.in_bytes[k], 256);
         p.out_off[k] = off; off += round_up(p.out_bytes[k], 256);
+        p.mask_off[k] = off; if (d.right_mode) off += round_up((size_t)d.n, 256);
     }
     p.results_off = off; off += round_up(sizeof(lgn_layer_result_t) * (size_t)L, 256);
     WsLayout w;
@@ -840,6 +925,12 @@ extern "C" lgn_status lgn_compress_layers_host(const lgn_layer_t *layers, int nu
         if (p.in_bytes[k] &&
             cudaMemcpyAsync(base + p.in_off[k], layers[k].g, p.in_bytes[k], cudaMemcpyHostToDevice, st) != cudaSuccess)
             return LGN_ERR_CUDA;
+        if (layers[k].right_mode) {
+            dev_layers[k].right_mode = base + p.mask_off[k];
+            if (layers[k].n &&
+                cudaMemcpyAsync(base + p.mask_off[k], layers[k].right_mode, (size_t)layers[k].n, cudaMemcpyHostToDevice, st) != cudaSuccess)
+                return LGN_ERR_CUDA;
+        }
     }
     lgn_layer_result_t *res_dev = reinterpret_cast<lgn_layer_result_t *>(base + p.results_off);
     lgn_status s = lgn_compress_layers(dev_layers.data(), num_layers, res_dev, base + p.ws_off, p.ws_bytes, stream);

@@ -53,16 +53,24 @@ dequantize_kernel(const uint32_t *__restrict__ codes, void *__restrict__ out, ui
     constexpr int NW = (kChunkBits + 31) / 32;                  // words that hold a chunk's codes once aligned
     __shared__ uint32_t sm[kTileWords + 4];                     // + words a chunk's window may reach past the tile
 
-    for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    // the next tile's code words are fetched into registers while the current tile is decoded
+    uint32_t r_next[NBITS];
+    auto fetch = [&](uint32_t tile) {
         const uint64_t w0 = (uint64_t)tile * kTileWords;
-        __syncthreads();                                        // the previous tile has been decoded
         #pragma unroll
         for (int k = 0; k < NBITS; ++k) {
-            const int idx = k * kThreads + threadIdx.x;
-            sm[idx] = (w0 + idx < total_words) ? __ldcs(codes + w0 + idx) : 0u;
+            const uint64_t w = w0 + (uint64_t)(k * kThreads + threadIdx.x);
+            r_next[k] = (tile < ntiles && w < total_words) ? __ldcs(codes + w) : 0u;
         }
+    };
+    fetch(blockIdx.x);
+    for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        __syncthreads();                                        // the previous tile has been decoded
+        #pragma unroll
+        for (int k = 0; k < NBITS; ++k) sm[k * kThreads + threadIdx.x] = r_next[k];
         if (threadIdx.x < 4) sm[kTileWords + threadIdx.x] = 0u;
         __syncthreads();
+        fetch(tile + gridDim.x);
 
         const uint64_t tile_base = (uint64_t)tile * kDqTileElems;
         const bool full = tile_base + kDqTileElems <= n;

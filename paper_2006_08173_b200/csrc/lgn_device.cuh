@@ -233,6 +233,8 @@ __device__ __forceinline__ float lg2_scaled(float a) {
 struct StatsAcc {            // per thread, in log2 units
     double s1 = 0.0, s2 = 0.0;
     unsigned long long cnt = 0;
+    unsigned long long right = 0;   // extended pass only: entries of the right mode (mask byte != 0)
+    float amax = 0.f;               // extended pass only: largest magnitude of the whole tensor
 };
 
 // Adds one tile to the thread's accumulators.  y = log2|x| + 24 in fp32.  The sums
@@ -289,27 +291,114 @@ __device__ __forceinline__ void stats_tile(const void *g, uint64_t tile_base, ui
     }
 }
 
+// The extended statistics tile: what stats_tile computes, restricted to the
+// entries whose byte in `mask` is non-zero when MASKED (the right mode of a
+// bi-modal gradient; the appendix's steps 1 and 3), plus the number of such
+// entries and the largest magnitude of the whole tile (Algorithm 1's max|X|).
+// Same pivoted sums as stats_tile.  Serves whole and ragged tiles; one chunk per
+// load step with the next step's loads issued before the current one is used.
+// The mask bytes of a chunk are the C bytes at the chunk's element index.
+template <int DT>
+__device__ __forceinline__ void load_mask_chunk(const uint8_t *mask, uint64_t i, uint64_t n, uint32_t (&m)[4]) {
+    constexpr int C = ElemTraits<DT>::kChunk;
+    m[0] = m[1] = m[2] = m[3] = 0u;
+    if (i + C <= n) {
+        if (C == 8) { const uint2 v = __ldg(reinterpret_cast<const uint2 *>(mask + i)); m[0] = v.x; m[1] = v.y; }
+        else        { const uint4 v = __ldg(reinterpret_cast<const uint4 *>(mask + i)); m[0] = v.x; m[1] = v.y; m[2] = v.z; m[3] = v.w; }
+    } else {
+        #pragma unroll
+        for (int k = 0; k < C; ++k) if (i + k < n) m[k >> 2] |= (uint32_t)mask[i + k] << ((k & 3) * 8);
+    }
+}
+
+template <int DT, bool MASKED>
+__device__ __forceinline__ void stats_tile_ext(const void *g, const uint8_t *mask, uint64_t tile_base, uint64_t n,
+                                               StatsAcc &acc) {
+    constexpr int C = ElemTraits<DT>::kChunk;
+    constexpr int kLoads = kTileElems / (kThreads * C);
+    const float kUnset = -__int_as_float(0x7F800000);
+    float P = kUnset, amax = 0.f;
+    double D1 = 0.0, D2 = 0.0;
+    unsigned long long Cn = 0, Rn = 0;
+    auto at = [&](int j) { return tile_base + (uint64_t)(j * kThreads + threadIdx.x) * C; };
+    Chunk cur = load_chunk<DT, false, Ld::Keep>(g, at(0), n), nxt = cur;
+    uint32_t mcur[4] = {~0u, ~0u, ~0u, ~0u}, mnxt[4] = {~0u, ~0u, ~0u, ~0u};
+    if (MASKED) load_mask_chunk<DT>(mask, at(0), n, mcur);
+    #pragma unroll 1
+    for (int j = 0; j < kLoads; ++j) {
+        if (j + 1 < kLoads) {
+            nxt = load_chunk<DT, false, Ld::Keep>(g, at(j + 1), n);
+            if (MASKED) load_mask_chunk<DT>(mask, at(j + 1), n, mnxt);
+        }
+        float y[C];
+        bool in[C];
+        #pragma unroll
+        for (int e = 0; e < C; ++e) {
+            const float a = fabsf(u2f(elem_bits<DT>(cur, e)));
+            amax = fmaxf(amax, a);
+            y[e] = lg2_scaled(a);
+            const bool right = !MASKED || ((mcur[e >> 2] >> ((e & 3) * 8)) & 0xFFu) != 0u;
+            if (MASKED) Rn += right ? 1u : 0u;
+            in[e] = right && y[e] != kUnset;
+        }
+        if (P == kUnset) {
+            #pragma unroll
+            for (int e = 0; e < C; ++e) if (in[e]) P = fmaxf(P, y[e]);
+        }
+        float s1 = 0.f, s2 = 0.f, cf = 0.f;
+        #pragma unroll
+        for (int e = 0; e < C; ++e) {
+            if (in[e]) {
+                const float d = y[e] - P;
+                s1 += d;
+                s2 = fmaf(d, d, s2);
+                cf += 1.0f;
+            }
+        }
+        D1 += (double)s1;
+        D2 += (double)s2;
+        Cn += (uint32_t)cf;
+        cur = nxt;
+        #pragma unroll
+        for (int k = 0; k < 4; ++k) mcur[k] = mnxt[k];
+    }
+    if (Cn) {
+        const double p = (double)P - (double)kLogShift, c = (double)Cn;
+        acc.s1 += D1 + c * p;
+        acc.s2 += D2 + p * (2.0 * D1 + c * p);
+        acc.cnt += Cn;
+    }
+    acc.right += Rn;
+    acc.amax = fmaxf(acc.amax, amax);
+}
+
 // Fixed-shape tree over the CTA; the result is valid in thread 0.
-__device__ __forceinline__ void block_reduce(StatsAcc &acc, double *sm /* 3*kWarps */) {
-    #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
+__device__ __forceinline__ void warp_reduce(StatsAcc &acc, int width) {
+    for (int off = width / 2; off > 0; off >>= 1) {
         acc.s1 += __shfl_down_sync(0xFFFFFFFFu, acc.s1, off);
         acc.s2 += __shfl_down_sync(0xFFFFFFFFu, acc.s2, off);
         acc.cnt += __shfl_down_sync(0xFFFFFFFFu, acc.cnt, off);
+        acc.right += __shfl_down_sync(0xFFFFFFFFu, acc.right, off);
+        acc.amax = fmaxf(acc.amax, __shfl_down_sync(0xFFFFFFFFu, acc.amax, off));
     }
+}
+
+__device__ __forceinline__ void block_reduce(StatsAcc &acc, double *sm /* 5*kWarps */) {
+    warp_reduce(acc, 32);
     const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
     __syncthreads();                      // sm may still be in use by an earlier reduction
-    if (l == 0) { sm[w] = acc.s1; sm[kWarps + w] = acc.s2; sm[2 * kWarps + w] = __longlong_as_double((long long)acc.cnt); }
+    if (l == 0) {
+        sm[w] = acc.s1; sm[kWarps + w] = acc.s2; sm[2 * kWarps + w] = __longlong_as_double((long long)acc.cnt);
+        sm[3 * kWarps + w] = __longlong_as_double((long long)acc.right); sm[4 * kWarps + w] = (double)acc.amax;
+    }
     __syncthreads();
     if (w == 0) {
         StatsAcc t;
-        if (l < kWarps) { t.s1 = sm[l]; t.s2 = sm[kWarps + l]; t.cnt = (unsigned long long)__double_as_longlong(sm[2 * kWarps + l]); }
-        #pragma unroll
-        for (int off = kWarps / 2; off > 0; off >>= 1) {
-            t.s1 += __shfl_down_sync(0xFFFFFFFFu, t.s1, off);
-            t.s2 += __shfl_down_sync(0xFFFFFFFFu, t.s2, off);
-            t.cnt += __shfl_down_sync(0xFFFFFFFFu, t.cnt, off);
+        if (l < kWarps) {
+            t.s1 = sm[l]; t.s2 = sm[kWarps + l]; t.cnt = (unsigned long long)__double_as_longlong(sm[2 * kWarps + l]);
+            t.right = (unsigned long long)__double_as_longlong(sm[3 * kWarps + l]); t.amax = (float)sm[4 * kWarps + l];
         }
+        warp_reduce(t, kWarps);
         acc = t;
     }
 }

@@ -8,13 +8,10 @@
 // the code words of its elements follow one another in index order, stream bit k
 // in bit (k mod 32) of word (k div 32), the FP value least-significant bit first.
 //
-// Three launches per call:
-//   count  every block's length in words                      (reads the tensor)
-//   scan   exclusive prefix sum of the lengths -> off[]       (one CTA)
-//   emit   code words again, each thread ORs its bits into the block's image in
-//          shared memory, whole words go out coalesced         (reads the tensor)
-// The pruning decisions are recomputed in `emit` from the same counter-based
-// random bits rather than stored in between.
+// One pass over the tensor (a memset of the small workspace, then one launch): each
+// CTA encodes whole blocks into an image in shared memory, obtains the block's
+// first word by a decoupled look-back over the lengths the preceding blocks have
+// published, and writes the image out with coalesced stores.
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -31,6 +28,7 @@ constexpr int kPfxThreads = 256;
 constexpr int kPfxPerThread = 8;                               // one block of random bits per thread
 static_assert(kPfxThreads * kPfxPerThread == (int)LGN_PREFIX_BLOCK, "a CTA pass covers one block");
 constexpr int kPfxWarps = kPfxThreads / 32;
+constexpr int kPfxImageWords = (LGN_PREFIX_BLOCK * 34u + 31u) / 32u + 4u;   // a block of FP values, plus slack
 
 template <int DT> struct PfxTraits;
 template <> struct PfxTraits<LGN_F32>  { static constexpr int kWidth = 32; static constexpr uint32_t kSign = 0x80000000u; };
@@ -89,199 +87,182 @@ __device__ __forceinline__ void pfx_values(uint32_t (&p)[kPfxPerThread], uint64_
     }
 }
 
-// Code word of one stored pattern: its bits (first stream bit in bit 0) and its
-// length.  An FP value is returned as the two prefix bits; the caller appends
-// the pattern.
-template <int DT>
-__device__ __forceinline__ uint32_t pfx_len(uint32_t pat, uint32_t tau_pat) {
-    if (pat == 0u) return 1u;
-    if (tau_pat != 0u && (pat & ~PfxTraits<DT>::kSign) == tau_pat) return 3u;
-    return 2u + PfxTraits<DT>::kWidth;
-}
-
 template <int DT>
 __device__ __forceinline__ uint32_t tau_pattern(float tau) {
     return DT == LGN_F32 ? f2u(tau) : f2u(tau) >> 16;
 }
 
+// ------------------------------------------------------------------ single-pass encoder
+// Blocks are handed out in index order by a ticket counter, so every block a CTA
+// may have to wait for is already in the hands of a running CTA.  Per block:
+//   1. load, prune (Eq. 5), classify; every thread assembles the short codes of its
+//      eight elements ("0", "100"/"101", or the "11" in front of a value: at most 24
+//      bits) in one register and notes where the values cut that string;
+//   2. a scan of the threads' bit counts over the CTA gives each thread's position
+//      and the block's length in words, which is published as this block's
+//      AGGREGATE;
+//   3. the threads OR their bits into the block's image in shared memory: for each
+//      value one 64-bit piece (the short bits since the previous value, then the
+//      value), then the remaining short bits;
+//   4. meanwhile warp 0 looks back over the preceding blocks' published lengths
+//      (decoupled look-back: an INCLUSIVE prefix ends the walk) to get the block's
+//      first word, publishes its own inclusive prefix, and the image goes out with
+//      coalesced stores.
+// Waits in the look-back are bounded; if one runs out every CTA stops and
+// off[nblocks] is set to all ones.
+struct PfxCtl { uint32_t ticket, error, pad[62]; };
+static_assert(sizeof(PfxCtl) == 256, "control block");
+constexpr unsigned long long kPfxAggregate = 1ull, kPfxInclusive = 2ull;
+constexpr uint32_t kPfxMaxPolls = 1u << 20;
+
+__device__ __forceinline__ unsigned long long ld_acquire64(const unsigned long long *p) {
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release64(unsigned long long *p, unsigned long long v) {
+    asm volatile("st.release.gpu.global.u64 [%0], %1;" :: "l"(p), "l"(v) : "memory");
+}
+
+// OR the low `len` bits of x (its other bits are zero) into the image at bit position `at`.
+__device__ __forceinline__ void pfx_or64(uint32_t *img, uint32_t at, unsigned long long x) {
+    const uint32_t s = at & 31u, w = at >> 5;
+    const uint32_t lo = (uint32_t)x, hi = (uint32_t)(x >> 32);
+    const uint32_t w0 = lo << s, w1 = __funnelshift_l(lo, hi, s), w2 = __funnelshift_l(hi, 0u, s);
+    if (w0) atomicOr(img + w, w0);
+    if (w1) atomicOr(img + w + 1, w1);
+    if (w2) atomicOr(img + w + 2, w2);
+}
+__device__ __forceinline__ void pfx_or32(uint32_t *img, uint32_t at, uint32_t x) {
+    const uint32_t s = at & 31u, w = at >> 5;
+    const uint32_t w0 = x << s, w1 = __funnelshift_l(x, 0u, s);
+    if (w0) atomicOr(img + w, w0);
+    if (w1) atomicOr(img + w + 1, w1);
+}
+
 template <int DT, bool PRUNE>
 __global__ void __launch_bounds__(kPfxThreads)
-prefix_count_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host, const lgn_layer_result_t *tau_from,
-                    uint64_t seed, Weyl wy, uint32_t *block_words) {
-    __shared__ uint32_t sm_total[2];
-    const float tau = pfx_tau(tau_host, tau_from);
-    const uint32_t tp = tau_pattern<DT>(tau);
-    if (threadIdx.x < 2) sm_total[threadIdx.x] = 0u;
-    __syncthreads();
-    uint32_t p[kPfxPerThread], q[kPfxPerThread];
-    uint64_t b = blockIdx.x;
-    if (b < nblocks) pfx_load<DT>(g, b * LGN_PREFIX_BLOCK + (uint64_t)threadIdx.x * kPfxPerThread, n, p);
-    for (uint32_t it = 0; b < nblocks; b += gridDim.x, ++it) {
-        const uint64_t i = b * LGN_PREFIX_BLOCK + (uint64_t)threadIdx.x * kPfxPerThread;
-        const uint64_t bn = b + gridDim.x;                       // the next block's loads fly while this one is counted
-        if (bn < nblocks) pfx_load<DT>(g, bn * LGN_PREFIX_BLOCK + (uint64_t)threadIdx.x * kPfxPerThread, n, q);
-        pfx_values<DT, PRUNE>(p, i, tau, seed, wy);
-        uint32_t bits = 0u;
-        if ((b + 1) * LGN_PREFIX_BLOCK <= n) {                   // the whole block lies inside the tensor
-            #pragma unroll
-            for (int k = 0; k < 8; ++k) bits += pfx_len<DT>(p[k], tp);
-        } else {
-            #pragma unroll
-            for (int k = 0; k < 8; ++k) if (i + k < n) bits += pfx_len<DT>(p[k], tp);
-        }
-        bits = __reduce_add_sync(0xFFFFFFFFu, bits);
-        if ((threadIdx.x & 31) == 0) atomicAdd(&sm_total[it & 1], bits);
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            block_words[b] = (sm_total[it & 1] + 31u) >> 5;
-            sm_total[it & 1] = 0u;                               // used again two blocks on, after the next barrier
-        }
-        #pragma unroll
-        for (int k = 0; k < 8; ++k) p[k] = q[k];
-    }
-}
-
-// Exclusive prefix sum of block_words[0..nblocks) into off[0..nblocks]; one CTA.
-// Thread t owns the entries [t*per, (t+1)*per), per a multiple of 4 (16-byte loads).
-constexpr int kScanThreads = 1024;
-__global__ void __launch_bounds__(kScanThreads)
-prefix_scan_kernel(const uint32_t *block_words, uint64_t nblocks, uint64_t *off) {
-    __shared__ unsigned long long sm[kScanThreads / 32];
-    const uint64_t per = ((nblocks + kScanThreads - 1) / kScanThreads + 3) / 4 * 4;
-    const uint64_t lo = (uint64_t)threadIdx.x * per < nblocks ? (uint64_t)threadIdx.x * per : nblocks;
-    const uint64_t hi = lo + per < nblocks ? lo + per : nblocks;
-    unsigned long long s = 0;
-    uint64_t k = lo;
-    for (; k + 4 <= hi; k += 4) {                                // lo is a multiple of 4: aligned
-        const uint4 v = *reinterpret_cast<const uint4 *>(block_words + k);
-        s += (unsigned long long)v.x + v.y + v.z + v.w;
-    }
-    for (; k < hi; ++k) s += block_words[k];
-    // inclusive scan of s over the CTA: warp shuffles, then the 32 warp totals
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    unsigned long long incl = s;
-    #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const unsigned long long v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-        if (lane >= d) incl += v;
-    }
-    if (lane == 31) sm[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        unsigned long long w = sm[lane];
-        #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const unsigned long long v = __shfl_up_sync(0xFFFFFFFFu, w, d);
-            if (lane >= d) w += v;
-        }
-        sm[lane] = w;                                            // inclusive over warps
-    }
-    __syncthreads();
-    unsigned long long run = incl - s + (warp ? sm[warp - 1] : 0ull);
-    for (k = lo; k + 4 <= hi; k += 4) {
-        const uint4 v = *reinterpret_cast<const uint4 *>(block_words + k);
-        off[k] = run; off[k + 1] = run + v.x; off[k + 2] = run + v.x + v.y; off[k + 3] = run + v.x + v.y + v.z;
-        run += (unsigned long long)v.x + v.y + v.z + v.w;
-    }
-    for (; k < hi; ++k) { off[k] = run; run += block_words[k]; }
-    if (threadIdx.x == kScanThreads - 1) off[nblocks] = sm[kScanThreads / 32 - 1];
-}
-
-constexpr int kPfxImageWords = (LGN_PREFIX_BLOCK * 34u + 31u) / 32u + 2u;   // a block of FP values, plus slack
-
-// A thread's code words, assembled in a 64-bit register that starts at the
-// thread's bit position inside its first image word; every completed 32-bit word
-// is ORed into the image (the first and last word of a thread are shared with its
-// neighbours; words that are all zero -- runs of "0" codes -- need no write).
-// nvalid = how many of the 8 elements exist (8 except in the tensor's last block).
-template <int DT>
-__device__ __forceinline__ void pfx_emit_thread(const uint32_t (&p)[kPfxPerThread], uint32_t tp, uint32_t pos,
-                                                uint32_t nvalid, uint32_t *img) {
+prefix_encode_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host, const lgn_layer_result_t *tau_from,
+                     uint64_t seed, Weyl wy, PfxCtl *ctl, unsigned long long *state, uint64_t *off, uint32_t *stream,
+                     uint64_t capacity_words) {
     constexpr uint32_t kSign = PfxTraits<DT>::kSign;
-    // Two 32-bit registers hold the bits from the current image word on; `tot` is
-    // the thread's bit position in the image.  Written without branches (selects
-    // and a predicated shared-memory OR): the lanes of a warp would take different
-    // paths at almost every element otherwise.
-    const uint32_t img_addr = (uint32_t)__cvta_generic_to_shared(img);
-    uint32_t lo = 0u, hi = 0u, tot = pos;
-    auto append = [&](uint32_t x, uint32_t len) {                // x has `len` bits; the low register has room
-        const uint32_t s = tot & 31u;
-        lo |= x << s;
-        hi |= __funnelshift_l(x, 0u, s);                         // x >> (32 - s), and 0 for s = 0
-        const uint32_t after = tot + len;
-        const uint32_t full = (after ^ tot) & 32u;               // the low register's word is complete
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\tsetp.ne.and.u32 p, %1, 0, p;\n\t"
-                     "@p red.shared.or.b32 [%0], %1;\n\t}"
-                     :: "r"(img_addr + (tot >> 5) * 4u), "r"(lo), "r"(full) : "memory");
-        lo = full ? hi : lo;
-        hi = full ? 0u : hi;
-        tot = after;
-    };
-    #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        const bool in = (uint32_t)k < nvalid;
-        const uint32_t pat = p[k];
-        const bool zero = pat == 0u;
-        const bool alpha = tp != 0u && (pat & ~kSign) == tp;
-        const bool value = in && !zero && !alpha;
-        const uint32_t v = zero ? 0u : alpha ? ((pat & kSign) ? 5u : 1u) : 3u;       // first stream bit in bit 0
-        append(in ? v : 0u, !in ? 0u : zero ? 1u : alpha ? 3u : 2u);
-        append(value ? pat : 0u, value ? (uint32_t)PfxTraits<DT>::kWidth : 0u);
-    }
-    if (lo) atomicOr(&img[tot >> 5], lo);
-}
-
-template <int DT, bool PRUNE>
-__global__ void __launch_bounds__(kPfxThreads)
-prefix_emit_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host, const lgn_layer_result_t *tau_from,
-                   uint64_t seed, Weyl wy, const uint64_t *off, uint32_t *stream, uint64_t capacity_words) {
+    constexpr uint32_t W = PfxTraits<DT>::kWidth;
     __shared__ uint32_t img[kPfxImageWords];
-    __shared__ uint32_t sm[kPfxWarps];
+    __shared__ uint32_t sm_scan[kPfxWarps];
+    __shared__ unsigned long long sm_ticket, sm_excl;
     const float tau = pfx_tau(tau_host, tau_from);
     const uint32_t tp = tau_pattern<DT>(tau);
+    const uint32_t tpc = tp ? tp : kSign;                        // a pattern no magnitude equals: no alpha codes when alpha = 0
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t p[kPfxPerThread], q[kPfxPerThread];
-    if (blockIdx.x < nblocks)
-        pfx_load<DT>(g, (uint64_t)blockIdx.x * LGN_PREFIX_BLOCK + (uint64_t)threadIdx.x * kPfxPerThread, n, p);
-    for (uint64_t b = blockIdx.x; b < nblocks; b += gridDim.x) {
-        const uint64_t w0 = off[b], w1 = off[b + 1];
-        const uint32_t words = (uint32_t)(w1 - w0);
+
+    for (;;) {
+        if (threadIdx.x == 0) sm_ticket = atomicAdd(&ctl->ticket, 1u);
+        __syncthreads();                                         // also: the previous block's image has gone out
+        const uint64_t b = sm_ticket;
+        if (b >= nblocks) break;
         const uint64_t i = b * LGN_PREFIX_BLOCK + (uint64_t)threadIdx.x * kPfxPerThread;
-        const uint64_t bn = b + gridDim.x;                       // the next block's loads fly while this one is packed
-        if (bn < nblocks) pfx_load<DT>(g, bn * LGN_PREFIX_BLOCK + (uint64_t)threadIdx.x * kPfxPerThread, n, q);
-        if (w1 > capacity_words) {                               // does not fit: the caller sees off[nblocks] > capacity
-            #pragma unroll
-            for (int k = 0; k < 8; ++k) p[k] = q[k];
-            continue;
-        }
-        for (uint32_t k = threadIdx.x; k < words + 1u; k += kPfxThreads) img[k] = 0u;
+        uint32_t p[kPfxPerThread];
+        pfx_load<DT>(g, i, n, p);
         pfx_values<DT, PRUNE>(p, i, tau, seed, wy);
-        const bool full = (b + 1) * LGN_PREFIX_BLOCK <= n;
-        const uint32_t nvalid = full ? 8u : (i >= n ? 0u : (n - i < 8u ? (uint32_t)(n - i) : 8u));
-        uint32_t bits = 0u;
+        const uint32_t nvalid = i >= n ? 0u : (n - i < 8u ? (uint32_t)(n - i) : 8u);
+
+        // short codes of the eight elements, first stream bit in bit 0
+        uint32_t sb = 0u, q = 0u, vm = 0u;
+        unsigned long long cuts = 0ull;                          // 5 bits per element: q after the element
         #pragma unroll
-        for (int k = 0; k < 8; ++k) if ((uint32_t)k < nvalid) bits += pfx_len<DT>(p[k], tp);
-        // exclusive scan of `bits` over the CTA: warp scan, then the warp totals
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t pat = p[k];
+            const bool in = (uint32_t)k < nvalid;
+            const bool nz = in && pat != 0u;
+            const bool al = in && (pat & ~kSign) == tpc;
+            const uint32_t code = al ? ((pat & kSign) ? 5u : 1u) : (nz ? 3u : 0u);
+            sb |= code << q;
+            q += (in ? 1u : 0u) + (nz ? 1u : 0u) + (al ? 1u : 0u);
+            if (nz && !al) vm |= 1u << k;
+            cuts |= (unsigned long long)q << (5 * k);
+        }
+        const uint32_t bits = q + W * __popc(vm);
+
+        // exclusive scan of `bits` over the CTA
         uint32_t incl = bits;
         #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, d);
             if (lane >= d) incl += v;
         }
-        if (lane == 31) sm[warp] = incl;
-        __syncthreads();                                         // also: the image is zeroed
-        uint32_t pos = incl - bits;
-        #pragma unroll
-        for (int w = 0; w < kPfxWarps; ++w) if (w < warp) pos += sm[w];
-        if (full) pfx_emit_thread<DT>(p, tp, pos, 8u, img);
-        else      pfx_emit_thread<DT>(p, tp, pos, nvalid, img);
+        if (lane == 31) sm_scan[warp] = incl;
         __syncthreads();
-        for (uint32_t k = threadIdx.x; k < words; k += kPfxThreads) stream[w0 + k] = img[k];
-        __syncthreads();                                         // the image and sm are reused by the next block
+        uint32_t pos = incl - bits, total = 0u;
         #pragma unroll
-        for (int k = 0; k < 8; ++k) p[k] = q[k];
+        for (int w = 0; w < kPfxWarps; ++w) { const uint32_t t = sm_scan[w]; if (w < warp) pos += t; total += t; }
+        const uint32_t words = (total + 31u) >> 5;
+        if (threadIdx.x == 0) {
+            if (b == 0) { st_release64(state, ((unsigned long long)words << 2) | kPfxInclusive); sm_excl = 0ull; }
+            else        st_release64(state + b, ((unsigned long long)words << 2) | kPfxAggregate);
+        }
+        for (uint32_t k = threadIdx.x; k < words + 2u; k += kPfxThreads) img[k] = 0u;
+        __syncthreads();
+
+        // the thread's bits into the image
+        uint32_t cur = pos, done = 0u;
+        #pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            if (vm & (1u << k)) {
+                const uint32_t cut = (uint32_t)(cuts >> (5 * k)) & 31u;
+                const uint32_t plen = cut - done;                // 2..26: ends with the value's "11"
+                const uint32_t piece = (sb >> done) & ((1u << plen) - 1u);
+                pfx_or64(img, cur, (unsigned long long)piece | ((unsigned long long)p[k] << plen));
+                cur += plen + W;
+                done = cut;
+            }
+        }
+        if (q > done) pfx_or32(img, cur, sb >> done);
+
+        // warp 0: first word of this block = sum of the lengths of all earlier blocks
+        if (warp == 0 && b > 0) {
+            unsigned long long excl = 0ull;
+            bool fail = false;
+            for (long long j = (long long)b - 1;; j -= 32) {
+                const long long idx = j - lane;
+                unsigned long long v = kPfxInclusive;            // before block 0: an inclusive prefix of 0
+                uint32_t polls = 0;
+                for (;;) {
+                    if (idx >= 0) v = ld_acquire64(state + idx);
+                    if (!__any_sync(0xFFFFFFFFu, (v & 3ull) == 0ull)) break;
+                    const bool stop = ++polls > kPfxMaxPolls || *(volatile uint32_t *)&ctl->error != 0u;
+                    if (__any_sync(0xFFFFFFFFu, stop)) { fail = true; break; }
+                    __nanosleep(64);
+                }
+                if (fail) break;
+                const uint32_t inc_mask = __ballot_sync(0xFFFFFFFFu, (v & 3ull) == kPfxInclusive);
+                const int first = inc_mask ? __ffs(inc_mask) - 1 : 32;       // nearest block with an inclusive prefix
+                unsigned long long c = lane <= first ? (v >> 2) : 0ull;
+                #pragma unroll
+                for (int d = 16; d > 0; d >>= 1) c += __shfl_down_sync(0xFFFFFFFFu, c, d);
+                excl += __shfl_sync(0xFFFFFFFFu, c, 0);
+                if (inc_mask) break;
+            }
+            if (lane == 0) {
+                if (fail) { atomicExch(&ctl->error, 1u); sm_excl = ~0ull; }
+                else      { st_release64(state + b, ((excl + words) << 2) | kPfxInclusive); sm_excl = excl; }
+            }
+        }
+        __syncthreads();                                         // the image is complete, the offset known
+        const unsigned long long w0 = sm_excl;
+        if (w0 == ~0ull) {                                       // a wait ran out: tell the caller and stop
+            if (threadIdx.x == 0) off[nblocks] = ~0ull;
+            break;
+        }
+        if (threadIdx.x == 0) {
+            off[b] = w0;
+            if (b + 1 == nblocks) off[nblocks] = w0 + words;
+        }
+        if (w0 + words <= capacity_words)                        // else: the caller sees off[nblocks] > capacity
+            for (uint32_t k = threadIdx.x; k < words; k += kPfxThreads) stream[w0 + k] = img[k];
     }
 }
+
+__global__ void prefix_empty_kernel(uint64_t *off) { off[0] = 0ull; }
 
 // One thread decodes one block.
 template <int DT>
@@ -347,7 +328,7 @@ extern "C" uint64_t lgn_prefix_bound_words(uint64_t n, lgn_dtype dt) {
 }
 
 extern "C" size_t lgn_prefix_workspace_bytes(uint64_t n) {
-    return (size_t)((lgn_prefix_blocks(n) * 4 + 255) / 256 * 256 + 256);
+    return (size_t)(sizeof(PfxCtl) + (lgn_prefix_blocks(n) * 8 + 255) / 256 * 256);
 }
 
 extern "C" lgn_status lgn_prefix_encode(const void *g, uint64_t n, lgn_dtype dt, double tau, uint64_t seed,
@@ -363,24 +344,23 @@ extern "C" lgn_status lgn_prefix_encode(const void *g, uint64_t n, lgn_dtype dt,
     if (ws == nullptr || !aligned_to(ws, 16) || ws_bytes < lgn_prefix_workspace_bytes(n)) return LGN_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint64_t nb = lgn_prefix_blocks(n);
-    uint32_t *bw = static_cast<uint32_t *>(ws);
     const float tau_used = dt == LGN_BF16 ? snap_threshold_bf16(tau) : snap_threshold_f32(tau);
     const Weyl wy = { kWeyl0, kWeyl1 };
-    if (nb > 0) {
-        #define LGN_PFX1(K, D, P, ...) { const unsigned grid = resident_grid(K<D, P>, nb); \
-                                         if (grid == 0) return LGN_ERR_CUDA; \
-                                         K<D, P><<<grid, kPfxThreads, 0, st>>>(__VA_ARGS__); }
-        #define LGN_PFX(K, ...) \
-            if (dt == LGN_F32) { if (apply_prune) LGN_PFX1(K, LGN_F32, true, __VA_ARGS__) else LGN_PFX1(K, LGN_F32, false, __VA_ARGS__) } \
-            else               { if (apply_prune) LGN_PFX1(K, LGN_BF16, true, __VA_ARGS__) else LGN_PFX1(K, LGN_BF16, false, __VA_ARGS__) }
-        LGN_PFX(prefix_count_kernel, g, n, nb, tau_used, tau_from_dev, seed, wy, bw)
-        prefix_scan_kernel<<<1, kScanThreads, 0, st>>>(bw, nb, off_dev);
-        LGN_PFX(prefix_emit_kernel, g, n, nb, tau_used, tau_from_dev, seed, wy, off_dev, stream_dev, capacity_words)
-        #undef LGN_PFX
-        #undef LGN_PFX1
-    } else {
-        prefix_scan_kernel<<<1, kScanThreads, 0, st>>>(bw, 0, off_dev);
+    if (nb == 0) {
+        prefix_empty_kernel<<<1, 1, 0, st>>>(off_dev);
+        return cudaGetLastError() == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
     }
+    // ticket, error flag and the per-block look-back states start at zero
+    if (cudaMemsetAsync(ws, 0, lgn_prefix_workspace_bytes(n), st) != cudaSuccess) return LGN_ERR_CUDA;
+    PfxCtl *ctl = static_cast<PfxCtl *>(ws);
+    unsigned long long *state = reinterpret_cast<unsigned long long *>(static_cast<char *>(ws) + sizeof(PfxCtl));
+    #define LGN_PFX1(D, P) { const unsigned grid = resident_grid(prefix_encode_kernel<D, P>, nb); \
+                             if (grid == 0) return LGN_ERR_CUDA; \
+                             prefix_encode_kernel<D, P><<<grid, kPfxThreads, 0, st>>>(g, n, nb, tau_used, tau_from_dev, seed, wy, \
+                                 ctl, state, off_dev, stream_dev, capacity_words); }
+    if (dt == LGN_F32) { if (apply_prune) LGN_PFX1(LGN_F32, true) else LGN_PFX1(LGN_F32, false) }
+    else               { if (apply_prune) LGN_PFX1(LGN_BF16, true) else LGN_PFX1(LGN_BF16, false) }
+    #undef LGN_PFX1
     return cudaGetLastError() == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
 }
 

@@ -29,8 +29,8 @@ def test_every_declared_symbol_is_exported(lgn):
 def test_struct_sizes_match_header(lgn):
     assert C.sizeof(lgn.StatsT) == 48
     assert C.sizeof(lgn.FpFormatT) == 16
-    assert C.sizeof(lgn.LayerT) == 80
-    assert C.sizeof(lgn.LayerResultT) == 80
+    assert C.sizeof(lgn.LayerT) == 88
+    assert C.sizeof(lgn.LayerResultT) == 88
 
 
 def test_status_strings(lgn):
@@ -133,7 +133,7 @@ def test_device_entry_points_reject_bad_arguments_before_any_cuda_call(lgn):
     # grouped
     def layer(**kw):
         d = dict(g=A, out=B, n=100, dt=0, mode=0, S=0.8, nbits=6, rounding=0, seed=0,
-                 use_override=0, reserved=0, mu_override=0.0, sigma_override=0.0)
+                 use_override=0, scale_mode=0, mu_override=0.0, sigma_override=0.0, right_mode=None)
         d.update(kw)
         return lgn.LayerT(*[d[f[0]] for f in lgn.LayerT._fields_])
     def call(l, ws_bytes=None, res=0x300000, n=1):
@@ -149,6 +149,11 @@ def test_device_entry_points_reject_bad_arguments_before_any_cuda_call(lgn):
     assert call(layer(g=A + 8)) == INVALID
     assert call(layer(use_override=1, sigma_override=-1.0)) == INVALID
     assert call(layer(use_override=1, mu_override=float("nan"), sigma_override=1.0)) == INVALID
+    assert call(layer(right_mode=0x400000 + 8)) == INVALID            # mask: 16-byte aligned
+    assert call(layer(right_mode=B + 16)) == INVALID                  # the output would overwrite the mask
+    assert call(layer(mode=1, right_mode=0x400000)) == INVALID        # a mask belongs to pruning
+    assert call(layer(scale_mode=1)) == INVALID                       # a scale mode belongs to quantisation
+    assert call(layer(mode=1, scale_mode=2)) == INVALID
     assert call(layer(), ws_bytes=16) == WORKSPACE
     assert call(layer(), res=None) == INVALID
     assert call(layer(), n=-1) == INVALID
@@ -173,3 +178,14 @@ def test_dequantize_rejects_bad_arguments_before_any_cuda_call(lgn):
     assert R.lgn_dequantize(A, 100, C.byref(ok), 0, A + 64, None) == INVALID                         # overlap
     assert R.lgn_dequantize(A, 2 ** 50, C.byref(ok), 0, B, None) == UNSUPPORTED
     assert R.lgn_dequantize(None, 0, C.byref(ok), 0, None, None) == 0                                # empty
+
+
+def test_scale_from_max(lgn, oracle):
+    for mx in [1.0, 1.0 - 2.0 ** -24, 3.0e-6, 2.0 ** -140, 1e4, 65504.0, 2.0 ** -20 * 1.5]:
+        for n2 in range(1, 8):
+            assert lgn.lgn_scale_from_max(mx, n2) == oracle.scale_exp_from_max(mx, n2)
+    for bad in [(0.0, 4), (-1.0, 4), (float("inf"), 4), (float("nan"), 4), (1.0, 0), (1.0, 8)]:
+        with pytest.raises(lgn.LgnError) as e:
+            lgn.lgn_scale_from_max(*bad)
+        assert e.value.code == 1
+    assert lgn.raw().lgn_scale_from_max(1.0, 4, None) == 1
