@@ -53,6 +53,14 @@ def _L():
         lib.orc_max_abs.restype = dbl
         lib.orc_scale_exp_from_max.argtypes = [dbl, i32]
         lib.orc_scale_exp_from_max.restype = i32
+        lib.orc_cosine_similarity.argtypes = [dbl, dbl, dbl]
+        lib.orc_cosine_similarity.restype = dbl
+        lib.orc_threshold_for_cosine.argtypes = [dbl, dbl, dbl]
+        lib.orc_threshold_for_cosine.restype = dbl
+        lib.orc_allocate_sparsity.argtypes = [i32, vp, vp, vp, vp, i32, vp, dbl, dbl, vp]
+        lib.orc_allocate_sparsity.restype = dbl
+        lib.orc_quantile_k.argtypes = [vp, u64, i32, dbl, dbl, dbl, C.POINTER(dbl)]
+        lib.orc_quantile_k.restype = dbl
         lib.orc_philox4x32.argtypes = [vp, vp, i32, vp]
         lib.orc_philox4x32.restype = None
         lib.orc_rand16.argtypes = [u64, u64]
@@ -222,6 +230,38 @@ def prune(g: np.ndarray, tau_used: float, seed: int, first: int = 0) -> np.ndarr
     out = np.empty_like(g)
     _L().orc_prune(_ptr(g), _ptr(out), g.size, _dtype_of(g), tau_used, seed, first)
     return out
+
+
+# --------------------------------------------------------------------------- cosine similarity / allocation
+def cosine_similarity(u: float, sigma: float, k: float) -> float:
+    """Expected cos between X and T(X) at threshold alpha = e^(mu+u), log cut off at k sigma."""
+    return float(_L().orc_cosine_similarity(u, sigma, k))
+
+
+def threshold_for_cosine(min_cos: float, sigma: float, k: float) -> float:
+    return float(_L().orc_threshold_for_cosine(min_cos, sigma, k))
+
+
+def allocate_sparsity(n, sigma, zero_frac, k, min_cos, S: float, s_max: float):
+    """Layers deepest first; the first len(min_cos) carry a cosine floor.  Returns
+    (per-layer sparsity list, element-weighted mean actually allocated)."""
+    L = len(n)
+    na = np.ascontiguousarray(n, dtype=np.uint64)
+    sa = np.ascontiguousarray(sigma, dtype=np.float64)
+    za = np.ascontiguousarray(zero_frac, dtype=np.float64)
+    ka = np.ascontiguousarray(k, dtype=np.float64)
+    ca = np.ascontiguousarray(list(min_cos) + [0.0], dtype=np.float64)
+    out = np.zeros(max(L, 1), dtype=np.float64)
+    mean = _L().orc_allocate_sparsity(L, _ptr(na), _ptr(sa), _ptr(za), _ptr(ka), len(min_cos), _ptr(ca), S, s_max, _ptr(out))
+    return [float(x) for x in out[:L]], float(mean)
+
+
+def quantile_k(g: np.ndarray, q: float, mu: float, sigma: float):
+    """(k, value): the q-quantile of ln|g| over the nonzeros in sigmas above mu, and the order statistic."""
+    g = _flat(g)
+    v = C.c_double()
+    k = _L().orc_quantile_k(_ptr(g), g.size, _dtype_of(g), q, mu, sigma, C.byref(v))
+    return float(k), v.value
 
 
 # --------------------------------------------------------------------------- format / quantize

@@ -32,6 +32,16 @@
  *                      powers of two and their neighbours by hand; the largest element's
  *                      exponent lands on E_max - 1 (checked with frexp in the test); no
  *                      element is clipped before rounding
+ *   orc_cosine_similarity
+ *                      Monte-Carlo: the measured cosine between a truncated lognormal sample
+ *                      and its stochastically pruned copy (orc_prune_one); alpha -> 0 gives 1;
+ *                      decreasing in alpha
+ *   orc_threshold_for_cosine
+ *                      inverse of the above (forward evaluation returns the target)
+ *   orc_allocate_sparsity
+ *                      hand-computed two- and three-layer budgets; the element-weighted mean of
+ *                      the result equals the requested overall sparsity; the cap; layers whose
+ *                      cosine is already above their floor keep the overall sparsity
  *   orc_dequantize     every code of every format against the value formula of Eq. 1-2
  *                      written out in the test; quantising the decoded value (nearest)
  *                      gives the code back
@@ -553,6 +563,151 @@ uint64_t orc_count_zeros(const void *g, uint64_t n, int dtype)
     uint64_t z = 0;
     for (uint64_t i = 0; i < n; ++i) z += (elem(g, dtype, i) == 0.0);
     return z;
+}
+
+/* ------------------------------------------------------------------ */
+/* Appendix "Cosine similarity and heterogeneous stochastic pruning"    */
+/* ------------------------------------------------------------------ */
+
+static double Phi(double z) { return 0.5 * erfc(-z / sqrt(2.0)); }
+
+/* Expected cosine of the angle between X and T_{alpha,eps}(X) for
+ * X ~ Lognormal(mu, sigma^2) whose logarithm is cut off k standard deviations above
+ * its mean (the appendix's three expectations; the lognormal is "truncated": the
+ * 0.997 quantile of the data stands in for the cut).  With u = ln(alpha / e^mu):
+ *
+ *   E[X.T(X)]  = E||X||^2 = n e^{2 s^2} Phi(k - 2 s)                          (a)
+ *   E||T(X)||^2 = n alpha e^{s^2/2} Phi((u - s^2)/s)
+ *               + n e^{2 s^2} [ Phi(k - 2 s) - Phi((u - 2 s^2)/s) ]           (b)
+ *   cos(theta) = (a) / sqrt((a) (b)) = sqrt((a)/(b))
+ *
+ * written with Phi(z) = 1/2 + 1/2 erf(z/rt2) for the printed erf terms; the scale
+ * e^mu cancels, so the formulas are those of the printed mu = 0 case at alpha/e^mu.
+ *
+ * Reading: the main text writes the cut as erf((k s - 2 s^2)/(s rt2)), i.e. ln x <= k s,
+ * while the step-by-step derivation writes ln(k s) in the same place.  The first is
+ * taken: k is "obtained from the distribution like sigma and mu" as a high quantile
+ * (0.997: the mass inside three standard deviations of a normal), which is a
+ * statement about ln x in units of sigma.  Zeros of the tensor add nothing to any of
+ * the three sums.  Requires u <= k s (a threshold above the cut prunes everything).
+ */
+double orc_cosine_similarity(double u, double sigma, double k)
+{
+    double s = sigma;
+    double top = Phi(k - 2.0 * s);
+    double a = exp(2.0 * s * s) * top;
+    double b = exp(u + 0.5 * s * s) * Phi((u - s * s) / s)
+             + exp(2.0 * s * s) * (top - Phi((u - 2.0 * s * s) / s));
+    if (!(b > 0.0)) return 1.0;
+    double c = sqrt(a / b);
+    return c > 1.0 ? 1.0 : c;
+}
+
+/* The largest u (threshold in units of e^mu, log scale) whose expected cosine is
+ * still >= min_cos; cos is 1 at u = -inf and falls as u grows.  Bisection on
+ * [-(40 s + 50), k s].  If even u = k s keeps the cosine above min_cos, returns k s. */
+double orc_threshold_for_cosine(double min_cos, double sigma, double k)
+{
+    double lo = -(40.0 * sigma + 50.0), hi = k * sigma;
+    if (orc_cosine_similarity(hi, sigma, k) >= min_cos) return hi;
+    for (int it = 0; it < 300; ++it) {
+        double mid = 0.5 * (lo + hi);
+        if (mid <= lo || mid >= hi) break;
+        if (orc_cosine_similarity(mid, sigma, k) >= min_cos) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+/* Inverse of orc_sparsity_of in u, by bisection (the same bracket as orc_threshold). */
+static double u_for_sparsity(double Sp, double sigma)
+{
+    double lo = -(40.0 * sigma + 50.0), hi = 40.0 * sigma + 50.0;
+    for (int it = 0; it < 300; ++it) {
+        double mid = 0.5 * (lo + hi);
+        if (mid <= lo || mid >= hi) break;
+        if (orc_sparsity_of(mid, sigma) < Sp) lo = mid; else hi = mid;
+    }
+    return 0.5 * (lo + hi);
+}
+
+/* Heterogeneous allocation (appendix "Heterogeneous algorithm").  Layers are given in
+ * backward-pass order, deepest first.  The first n_deep layers carry a floor
+ * min_cos[i] on their expected cosine similarity:
+ *   - at the overall sparsity S the layer's threshold is u_i (Eq. 8 with the layer's
+ *     zero fraction l_i, S' = (S - l_i)/(1 - l_i));
+ *   - if cos(u_i) < min_cos[i], the threshold is lowered to the one that reaches
+ *     the floor, and the layer's sparsity becomes l_i + (1 - l_i) F(u_i') (Eq. 8);
+ *   - otherwise it keeps S.
+ * The remaining layers share one level that restores the budget,
+ *   S_rest = (S * sum_all n_i - sum_deep n_i S_i) / sum_rest n_i,
+ * limited to s_max ("a maximum of 0.96-0.98 will prevent over-pruning") and to at
+ * least S.  out_S[i] receives every layer's sparsity.  Returns the element-weighted
+ * mean sparsity actually allocated (below S when the cap binds). */
+double orc_allocate_sparsity(int L, const uint64_t *n, const double *sigma, const double *zero_frac,
+                             const double *k, int n_deep, const double *min_cos,
+                             double S, double s_max, double *out_S)
+{
+    double total = 0.0, deep_elems = 0.0, deep_pruned = 0.0;
+    for (int i = 0; i < L; ++i) total += (double)n[i];
+    for (int i = 0; i < n_deep && i < L; ++i) {
+        double l = zero_frac[i], s = sigma[i];
+        double Si = S;
+        if (s < 1e-6) s = 1e-6;
+        if (l < 1.0 && S > l) {
+            double Sp = (S - l) / (1.0 - l);
+            double u = u_for_sparsity(Sp, s);
+            double cap = k[i] * s;
+            if (u > cap) u = cap;
+            if (orc_cosine_similarity(u, s, k[i]) < min_cos[i]) {
+                double u2 = orc_threshold_for_cosine(min_cos[i], s, k[i]);
+                Si = l + (1.0 - l) * orc_sparsity_of(u2, s);
+                if (Si > S) Si = S;
+            }
+        }
+        out_S[i] = Si;
+        deep_elems += (double)n[i];
+        deep_pruned += (double)n[i] * Si;
+    }
+    double rest = total - deep_elems;
+    double S_rest = S;
+    if (rest > 0.0) {
+        S_rest = (S * total - deep_pruned) / rest;
+        if (S_rest > s_max) S_rest = s_max;
+        if (S_rest < S) S_rest = S;
+    }
+    double pruned = deep_pruned;
+    for (int i = n_deep; i < L; ++i) { out_S[i] = S_rest; pruned += (double)n[i] * S_rest; }
+    return total > 0.0 ? pruned / total : 0.0;
+}
+
+/* The cut k of a tensor: the q-quantile of ln|g| over the nonzero entries, in standard
+ * deviations above the mean, k = (ln|g|_(r) - mu) / sigma with r = ceil(q * nnz) (1-based
+ * order statistic).  Also returns the order statistic itself through *value. */
+static int cmp_double(const void *a, const void *b)
+{
+    double x = *(const double *)a, y = *(const double *)b;
+    return (x > y) - (x < y);
+}
+
+double orc_quantile_k(const void *g, uint64_t n, int dtype, double q, double mu, double sigma, double *value)
+{
+    double *a = (double *)malloc((n ? n : 1) * sizeof(double));
+    uint64_t m = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        double x = fabs(elem(g, dtype, i));
+        if (x != 0.0) a[m++] = x;
+    }
+    double v = 0.0;
+    if (m) {
+        qsort(a, m, sizeof(double), cmp_double);
+        uint64_t r = (uint64_t)ceil(q * (double)m);
+        if (r < 1) r = 1;
+        if (r > m) r = m;
+        v = a[r - 1];
+    }
+    free(a);
+    if (value) *value = v;
+    return (m && sigma > 0.0) ? (log(v) - mu) / sigma : 0.0;
 }
 
 /* ------------------------------------------------------------------ */
