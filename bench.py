@@ -64,6 +64,12 @@ for _lg in (26, 28):
         WORKLOADS[f"dequant_fp6_to_{_odt}_2p{_lg}"] = dict(net="aux", kind="dequant", log2n=_lg, nbits=6,
                                                            dtype="f32" if _odt == "fp32" else "bf16", mode="dequant")
     for _dt in ("fp32", "bf16"):
+        WORKLOADS[f"bimodal_prune_{_dt}_2p{_lg}"] = dict(net="aux", kind="bimodal", log2n=_lg,
+                                                         dtype="f32" if _dt == "fp32" else "bf16", mode="prune")
+        WORKLOADS[f"max_scale_fp6_{_dt}_2p{_lg}"] = dict(net="aux", kind="maxscale", log2n=_lg, nbits=6,
+                                                         dtype="f32" if _dt == "fp32" else "bf16", mode="quant")
+        WORKLOADS[f"quantile_{_dt}_2p{_lg}"] = dict(net="aux", kind="quantile", log2n=_lg,
+                                                    dtype="f32" if _dt == "fp32" else "bf16", mode="quantile")
         WORKLOADS[f"prefix_encode_{_dt}_2p{_lg}"] = dict(net="aux", kind="prefix", log2n=_lg,
                                                          dtype="f32" if _dt == "fp32" else "bf16", mode="prefix")
 
@@ -356,6 +362,33 @@ def run_aux(args):
         alg_bytes = n * (w["nbits"] / 8.0 + esize)
         call = lambda: lgn.lgn_dequantize(codes, n, fmt, out)
         kernel = "dequantize_kernel"
+    elif w["kind"] == "quantile":
+        g = synth.lognormal_tensor(n, -12.0, 2.0, 0.5, 0, dtype, str(dev))
+        ws = torch.empty(lgn.lgn_quantile_workspace_bytes(), dtype=torch.uint8, device=dev)
+        out = torch.empty(16, dtype=torch.uint8, device=dev)
+        raw, gp, code, st_ = lgn.raw(), g.data_ptr(), lgn.dtype_code(g), torch.cuda.current_stream().cuda_stream
+        call = lambda: raw.lgn_quantile(gp, n, code, 0.997, out.data_ptr(), ws.data_ptr(), ws.numel(), st_)
+        alg_bytes = float(n * esize)                    # one read of the tensor (the fp32 selection reads it twice)
+        kernel = "quantile_top_kernel (+ quantile_low_kernel for fp32)"
+        launches = 5 if esize == 4 else 3
+    elif w["kind"] in ("bimodal", "maxscale"):
+        # one layer of the grouped call with the variant switched on
+        if w["kind"] == "bimodal":
+            g, mask = synth.bimodal_tensor(n, -9.0, 1.5, -17.0, 1.0, 0.5, 0, dtype, str(dev))
+            out = torch.empty_like(g)
+            layer = lgn.make_layer(g, out, lgn.MODE_PRUNE, S=0.85, seed=1, right_mode=mask)
+            alg_bytes = n * (3.0 * esize + 1.0)          # statistics read + mask, apply read, write
+        else:
+            g = synth.lognormal_tensor(n, -12.0, 2.0, 0.5, 0, dtype, str(dev))
+            out = torch.empty(lgn.lgn_codes_bytes(n, w["nbits"]), dtype=torch.uint8, device=dev)
+            layer = lgn.make_layer(g, out, lgn.MODE_QUANTIZE, nbits=w["nbits"], rounding=lgn.ROUND_STOCHASTIC, seed=1,
+                                   scale_mode=lgn.SCALE_FROM_MAX)
+            alg_bytes = n * (2.0 * esize + w["nbits"] / 8.0)
+        ws = lgn.new_workspace([n], dev)
+        res = lgn.new_results(1, dev)
+        call = lambda: lgn.lgn_compress_layers([layer], res, ws)
+        kernel = "compress_kernel"
+        launches = lgn.lgn_launches_per_call(1)
     else:
         g = synth.lognormal_tensor(n, -12.0, 2.0, 0.5, 0, dtype, str(dev))
         st = lgn.lgn_stats(g)
@@ -368,8 +401,8 @@ def run_aux(args):
         torch.cuda.synchronize()
         words = int(off_dev[-1].item())
         alg_bytes = n * esize + 4.0 * words          # one read of the tensor + the stream written
-        kernel = "prefix_count_kernel + prefix_scan_kernel + prefix_emit_kernel"
-        launches = 3
+        kernel = "prefix_encode_kernel"
+        launches = 1
     for _ in range(args.warmup):
         call()
     torch.cuda.synchronize()

@@ -113,6 +113,16 @@ size_t lgn_codes_bytes(uint64_t n, int nbits);
 lgn_status lgn_stats(const void *g, uint64_t n, lgn_dtype dt, lgn_stats_t *out_dev,
                      void *ws, size_t ws_bytes, void *stream);
 
+/* Statistics of the union of several tensors from the statistics of each: n, nnz,
+ * sum_ln and sum_ln2 add up; mu and sigma are formed from the totals.  This is the
+ * one exchange step of data-parallel training that wants the SAME threshold or format
+ * on every rank for a layer (each rank holds its own micro-batch slice of the
+ * gradient): the ranks all-reduce these four sums per layer (32 bytes) between the
+ * statistics pass and the closed form.  Host only.
+ *   parts  host array of nparts records (their mu and sigma fields are ignored)
+ *   out    host, receives the combined record */
+lgn_status lgn_combine_stats(const lgn_stats_t *parts, int nparts, lgn_stats_t *out);
+
 /* Sparsity -> threshold (Eq. 8 solved for alpha; Appendix A.9 steps 1-2).
  * Host only, no CUDA call.
  *   mu, sigma  lognormal parameters of the nonzero part
@@ -139,6 +149,51 @@ lgn_status lgn_fp_format(double mu, double sigma, int nbits, lgn_fp_format_t *fm
  * exponent bits: e_s = floor(log2 max_abs) - (2^(exp_bits-1) - 1).  Host only.
  * max_abs must be finite and > 0, exp_bits in 1..7. */
 lgn_status lgn_scale_from_max(double max_abs, int exp_bits, int32_t *scale_exp);
+
+/* ---- Cosine similarity and per-layer sparsity (appendix "Cosine similarity and
+ * heterogeneous stochastic pruning") ----
+ * lgn_cosine_similarity: the expected cosine of the angle between a layer's gradient and
+ * its stochastically pruned copy at threshold tau, for magnitudes whose logarithm is
+ * normal (mu, sigma) and cut off k standard deviations above mu ("the neural gradients'
+ * lognormal distributions are truncated"; k is the 0.997 quantile of the data in
+ * sigmas, lgn_quantile).  Host only.  tau must be > 0 and ln(tau) - mu <= k*sigma
+ * (a threshold above the cut prunes everything): otherwise LGN_ERR_INVALID_ARG. */
+lgn_status lgn_cosine_similarity(double mu, double sigma, double k, double tau, double *cosine);
+
+/* lgn_allocate_sparsity: the heterogeneous scheme.  Layers in backward-pass order,
+ * deepest first; the first num_deep of them carry a floor min_cos on the expected
+ * cosine similarity.  A deep layer whose cosine at the overall sparsity S is below its
+ * floor gets the lower sparsity at which the floor is met; the remaining layers share
+ * the one level that restores the element-weighted budget S, limited to s_max (the
+ * appendix suggests 0.96-0.98) and not below S.  Host only.
+ *   layers     host array; sigma, zero_frac, k of each layer from its statistics
+ *   S_out      host array of num_layers sparsities, to be used as lgn_layer_t.S
+ *   achieved   host, may be NULL: the element-weighted mean of S_out (below S when
+ *              the cap binds) */
+typedef struct {
+    uint64_t n;          /* elements                                                  */
+    double   sigma;      /* std of ln|g| over the nonzeros (clamped to [1e-6, 25])     */
+    double   zero_frac;  /* l, fraction of exact zeros                                */
+    double   k;          /* cut of the lognormal, in sigmas                            */
+    double   min_cos;    /* floor on the cosine similarity (deep layers only)          */
+} lgn_alloc_layer_t;
+lgn_status lgn_allocate_sparsity(const lgn_alloc_layer_t *layers, int num_layers, int num_deep,
+                                 double S, double s_max, double *S_out, double *achieved);
+
+/* lgn_quantile: the order statistic of rank ceil(q * nnz) (1-based) of |g| over the
+ * nonzero elements, exactly, by a radix selection on the magnitude patterns (one pass
+ * over a bf16 tensor, two over an fp32 tensor).  With the layer's mu and sigma,
+ * k = (ln(value) - mu) / sigma is the cut used above.
+ *   g        device, n elements of dt, 32-byte aligned
+ *   q        in [0, 1]
+ *   out_dev  device, 16 bytes, 16-byte aligned: { float value; uint32_t pad; uint64_t nnz }
+ *            (value 0 when the tensor has no nonzero element)
+ *   ws       device scratch of lgn_quantile_workspace_bytes() bytes, 16-byte aligned
+ * Three (bf16) or five (fp32) small launches on `stream`, no allocation. */
+typedef struct { float value; uint32_t pad; uint64_t nnz; } lgn_quantile_t;
+size_t     lgn_quantile_workspace_bytes(void);
+lgn_status lgn_quantile(const void *g, uint64_t n, lgn_dtype dt, double q, lgn_quantile_t *out_dev,
+                        void *ws, size_t ws_bytes, void *stream);
 
 /* Stochastic pruning with a given threshold (Eq. 5): the steady-state call
  * between refreshes of the statistics.

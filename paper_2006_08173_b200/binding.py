@@ -39,6 +39,15 @@ class FpFormatT(C.Structure):
                 ("scale_exp", C.c_int32)]
 
 
+class AllocLayerT(C.Structure):
+    _fields_ = [("n", C.c_uint64), ("sigma", C.c_double), ("zero_frac", C.c_double), ("k", C.c_double),
+                ("min_cos", C.c_double)]
+
+
+class QuantileT(C.Structure):
+    _fields_ = [("value", C.c_float), ("pad", C.c_uint32), ("nnz", C.c_uint64)]
+
+
 class LayerT(C.Structure):
     _fields_ = [("g", C.c_void_p), ("out", C.c_void_p), ("n", C.c_uint64),
                 ("dt", C.c_int32), ("mode", C.c_int32), ("S", C.c_double),
@@ -69,6 +78,16 @@ _lib.lgn_snap_threshold.argtypes = [_dbl, _i32]
 _lib.lgn_snap_threshold.restype = _dbl
 _lib.lgn_fp_format.argtypes = [_dbl, _dbl, _i32, C.POINTER(FpFormatT)]
 _lib.lgn_fp_format.restype = _i32
+_lib.lgn_cosine_similarity.argtypes = [_dbl, _dbl, _dbl, _dbl, C.POINTER(_dbl)]
+_lib.lgn_cosine_similarity.restype = _i32
+_lib.lgn_allocate_sparsity.argtypes = [C.POINTER(AllocLayerT), _i32, _i32, _dbl, _dbl, C.POINTER(_dbl), C.POINTER(_dbl)]
+_lib.lgn_allocate_sparsity.restype = _i32
+_lib.lgn_quantile_workspace_bytes.argtypes = []
+_lib.lgn_quantile_workspace_bytes.restype = _sz
+_lib.lgn_quantile.argtypes = [_vp, _u64, _i32, _dbl, _vp, _vp, _sz, _vp]
+_lib.lgn_quantile.restype = _i32
+_lib.lgn_combine_stats.argtypes = [C.POINTER(StatsT), _i32, C.POINTER(StatsT)]
+_lib.lgn_combine_stats.restype = _i32
 _lib.lgn_scale_from_max.argtypes = [_dbl, _i32, C.POINTER(C.c_int32)]
 _lib.lgn_scale_from_max.restype = _i32
 _lib.lgn_prune.argtypes = [_vp, _vp, _u64, _i32, _dbl, _u64, _vp]
@@ -173,6 +192,47 @@ def lgn_fp_format(mu: float, sigma: float, nbits: int) -> Dict[str, int]:
     f = FpFormatT()
     _check(_lib.lgn_fp_format(mu, sigma, nbits, C.byref(f)), "lgn_fp_format")
     return {"nbits": f.nbits, "exp_bits": f.exp_bits, "man_bits": f.man_bits, "scale_exp": f.scale_exp}
+
+
+def lgn_cosine_similarity(mu: float, sigma: float, k: float, tau: float) -> float:
+    c = _dbl()
+    _check(_lib.lgn_cosine_similarity(mu, sigma, k, tau, C.byref(c)), "lgn_cosine_similarity")
+    return c.value
+
+
+def lgn_allocate_sparsity(layers: Sequence[Dict[str, float]], num_deep: int, S: float, s_max: float):
+    """``layers``: dicts with n, sigma, zero_frac, k and (deep layers) min_cos, deepest first.
+    Returns (per-layer sparsity list, element-weighted mean allocated)."""
+    L = len(layers)
+    arr = (AllocLayerT * max(1, L))(*[AllocLayerT(int(a["n"]), float(a["sigma"]), float(a["zero_frac"]),
+                                                  float(a.get("k", 0.0)), float(a.get("min_cos", 0.0))) for a in layers])
+    out = (_dbl * max(1, L))()
+    mean = _dbl()
+    _check(_lib.lgn_allocate_sparsity(arr, L, num_deep, S, s_max, out, C.byref(mean)), "lgn_allocate_sparsity")
+    return [out[i] for i in range(L)], mean.value
+
+
+def lgn_quantile_workspace_bytes() -> int:
+    return int(_lib.lgn_quantile_workspace_bytes())
+
+
+def lgn_quantile(g: torch.Tensor, q: float, ws: Optional[torch.Tensor] = None, stream=None) -> Dict[str, float]:
+    """The order statistic of rank ceil(q nnz) of |g| over the nonzeros (synchronises to read it back)."""
+    ws = ws if ws is not None else torch.empty(lgn_quantile_workspace_bytes(), dtype=torch.uint8, device=g.device)
+    out = torch.empty(16, dtype=torch.uint8, device=g.device)
+    _check(_lib.lgn_quantile(_dev(g, "g") if g.numel() else None, g.numel(), dtype_code(g), float(q), _dev(out, "out"),
+                             _dev(ws, "ws"), ws.numel(), _stream(stream)), "lgn_quantile")
+    r = QuantileT.from_buffer_copy(out.cpu().numpy().tobytes())
+    return {"value": float(r.value), "nnz": int(r.nnz)}
+
+
+def lgn_combine_stats(parts: Sequence[Dict[str, float]]) -> Dict[str, float]:
+    """Statistics of the union of tensors from each one's n, nnz, sum_ln, sum_ln2."""
+    arr = (StatsT * max(1, len(parts)))(*[StatsT(int(p["n"]), int(p["nnz"]), float(p["sum_ln"]), float(p["sum_ln2"]),
+                                                 0.0, 0.0) for p in parts])
+    out = StatsT()
+    _check(_lib.lgn_combine_stats(arr, len(parts), C.byref(out)), "lgn_combine_stats")
+    return {"n": out.n, "nnz": out.nnz, "sum_ln": out.sum_ln, "sum_ln2": out.sum_ln2, "mu": out.mu, "sigma": out.sigma}
 
 
 def lgn_scale_from_max(max_abs: float, exp_bits: int) -> int:

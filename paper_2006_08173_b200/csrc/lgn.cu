@@ -354,8 +354,11 @@ constexpr int kAny = -1;                      // template value: decided per lay
 
 // DT, MODE, NBITS, SR fix what every layer of the group has in common, so that
 // the hot tile bodies are inlined and nothing else is compiled into the kernel;
-// kAny for all four is the general kernel for mixed groups.
-template <int DT, int MODE, int NBITS, int SR>
+// kAny for all four is the general kernel for mixed groups.  EXT: the group's
+// layers may ask for the extended statistics tile (a right-mode mask, max|g|);
+// every specialised kernel exists without and (as a second instance) with it, so a
+// group that does not ask pays nothing for it.
+template <int DT, int MODE, int NBITS, int SR, bool EXT = false>
 __global__ void __launch_bounds__(kThreads, kMinCtas)
 compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Segment *segs,
                 int num_layers, uint32_t total_items, Partial *partials) {
@@ -411,7 +414,7 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
         LayerDyn *D = dyn + sg.layer;
 
         if (sg.phase != kPhaseApply) {
-            const bool ext = sg.phase == kPhaseStatsExt;
+            const bool ext = (EXT || !kSpecial) && sg.phase == kPhaseStatsExt;
             if constexpr (kSpecial) {
                 run_stats_tile<DT, true>(L, tile, ext, partials, sm_red);
             } else {
@@ -479,19 +482,29 @@ quantize_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, const __g
 }
 
 // ------------------------------------------------------------------ kernel tables
-// variant index: 0 statistics only, 1 prune, 2 + 2*(nbits-4) + sr quantise
-constexpr int kVariants = 12;
+// variant index: 0 statistics only, 1 prune, 2 + 2*(nbits-4) + sr quantise; with extended
+// statistics: 12 prune, 13 + 2*(nbits-4) + sr quantise
+constexpr int kVariants = 23;
+constexpr int kVariantPruneExt = 12, kVariantQuantExt0 = 13;
 #define LGN_CK(DT, MODE, NB, SR) reinterpret_cast<const void *>(&compress_kernel<DT, MODE, NB, SR>)
+#define LGN_CKX(DT, MODE, NB, SR) reinterpret_cast<const void *>(&compress_kernel<DT, MODE, NB, SR, true>)
 #define LGN_CK_ROW(DT) { LGN_CK(DT, kModeStatsOnly, kAny, kAny), LGN_CK(DT, LGN_MODE_PRUNE, kAny, kAny), \
     LGN_CK(DT, LGN_MODE_QUANTIZE, 4, 0), LGN_CK(DT, LGN_MODE_QUANTIZE, 4, 1), \
     LGN_CK(DT, LGN_MODE_QUANTIZE, 5, 0), LGN_CK(DT, LGN_MODE_QUANTIZE, 5, 1), \
     LGN_CK(DT, LGN_MODE_QUANTIZE, 6, 0), LGN_CK(DT, LGN_MODE_QUANTIZE, 6, 1), \
     LGN_CK(DT, LGN_MODE_QUANTIZE, 7, 0), LGN_CK(DT, LGN_MODE_QUANTIZE, 7, 1), \
-    LGN_CK(DT, LGN_MODE_QUANTIZE, 8, 0), LGN_CK(DT, LGN_MODE_QUANTIZE, 8, 1) }
+    LGN_CK(DT, LGN_MODE_QUANTIZE, 8, 0), LGN_CK(DT, LGN_MODE_QUANTIZE, 8, 1), \
+    LGN_CKX(DT, LGN_MODE_PRUNE, kAny, kAny), \
+    LGN_CKX(DT, LGN_MODE_QUANTIZE, 4, 0), LGN_CKX(DT, LGN_MODE_QUANTIZE, 4, 1), \
+    LGN_CKX(DT, LGN_MODE_QUANTIZE, 5, 0), LGN_CKX(DT, LGN_MODE_QUANTIZE, 5, 1), \
+    LGN_CKX(DT, LGN_MODE_QUANTIZE, 6, 0), LGN_CKX(DT, LGN_MODE_QUANTIZE, 6, 1), \
+    LGN_CKX(DT, LGN_MODE_QUANTIZE, 7, 0), LGN_CKX(DT, LGN_MODE_QUANTIZE, 7, 1), \
+    LGN_CKX(DT, LGN_MODE_QUANTIZE, 8, 0), LGN_CKX(DT, LGN_MODE_QUANTIZE, 8, 1) }
 static const void *const kCompressTable[2][kVariants] = { LGN_CK_ROW(LGN_F32), LGN_CK_ROW(LGN_BF16) };
 static const void *const kCompressGeneral = LGN_CK(kAny, kAny, kAny, kAny);
 #undef LGN_CK_ROW
 #undef LGN_CK
+#undef LGN_CKX
 
 #define LGN_QK(DT, NB, SR) reinterpret_cast<const void *>(&quantize_kernel<DT, NB, SR>)
 #define LGN_QK_ROW(DT) { LGN_QK(DT, 4, 0), LGN_QK(DT, 4, 1), LGN_QK(DT, 5, 0), LGN_QK(DT, 5, 1), LGN_QK(DT, 6, 0), \
@@ -627,7 +640,6 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
     if (ws_bytes < w.total) return LGN_ERR_WORKSPACE;
 
     std::vector<LayerState> st(L);
-    uint32_t partial0 = 0;
     for (int k = 0; k < L; ++k) {
         const lgn_layer_t &d = layers[k].d;
         LayerState &s = st[k];
@@ -635,12 +647,33 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
         s.g = d.g; s.out = d.out; s.n = d.n; s.seed = d.seed; s.S = d.S;
         s.mu_override = d.mu_override; s.sigma_override = d.sigma_override;
         s.stats_out = layers[k].stats_out; s.result_out = layers[k].result_out;
-        s.ntiles = (uint32_t)((d.n + kTileElems - 1) / kTileElems);
-        s.partial0 = partial0;
         s.dt = d.dt; s.mode = d.mode; s.nbits = d.nbits; s.rounding = d.rounding;
         s.use_override = d.use_override ? 1 : 0;
         s.scale_mode = d.scale_mode;
         s.mask = static_cast<const uint8_t *>(d.right_mode);
+    }
+
+    // one kernel per (type, mode, width, rounding) shared by all layers; the general one otherwise.
+    // Extended statistics: the specialised kernels' second instances; mixed groups go general.
+    bool any_ext = false, same = true;
+    for (int k = 0; k < L; ++k) {
+        any_ext = any_ext || needs_ext_stats(st[k]);
+        same = same && st[k].dt == st[0].dt && variant_of(st[k].mode, st[k].nbits, st[k].rounding) ==
+                                                   variant_of(st[0].mode, st[0].nbits, st[0].rounding);
+    }
+    const void *fn = kCompressGeneral;
+    if (same && !any_ext) fn = kCompressTable[st[0].dt][variant_of(st[0].mode, st[0].nbits, st[0].rounding)];
+    else if (same && st[0].mode == LGN_MODE_PRUNE) fn = kCompressTable[st[0].dt][kVariantPruneExt];
+    else if (same && st[0].mode == LGN_MODE_QUANTIZE)
+        fn = kCompressTable[st[0].dt][kVariantQuantExt0 + variant_of(st[0].mode, st[0].nbits, st[0].rounding) - 2];
+    int grid = persistent_ctas(fn);
+    if (grid < 1) return LGN_ERR_CUDA;
+
+    uint32_t partial0 = 0;
+    for (int k = 0; k < L; ++k) {
+        LayerState &s = st[k];
+        s.ntiles = (uint32_t)((s.n + kTileElems - 1) / kTileElems);
+        s.partial0 = partial0;
         partial0 += s.ntiles;
     }
     std::vector<Segment> segs;
@@ -673,14 +706,6 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
     }
     if (cudaGetLastError() != cudaSuccess) return LGN_ERR_CUDA;
 
-    // one kernel per (type, mode, width, rounding) shared by all layers; the general one otherwise
-    const void *fn = kCompressTable[st[0].dt][variant_of(st[0].mode, st[0].nbits, st[0].rounding)];
-    for (int k = 1; k < L; ++k)
-        if (st[k].dt != st[0].dt || variant_of(st[k].mode, st[k].nbits, st[k].rounding) !=
-                                        variant_of(st[0].mode, st[0].nbits, st[0].rounding))
-            fn = kCompressGeneral;
-    int grid = persistent_ctas(fn);
-    if (grid < 1) return LGN_ERR_CUDA;
     if ((uint32_t)grid > total_items) grid = (int)(total_items ? total_items : 1u);
     WsHeader *a_hdr = reinterpret_cast<WsHeader *>(base);
     const LayerState *a_states = reinterpret_cast<const LayerState *>(base + w.states);
@@ -742,6 +767,25 @@ extern "C" lgn_status lgn_stats(const void *g, uint64_t n, lgn_dtype dt, lgn_sta
     return run_layers(std::vector<InternalLayer>(1, il), ws, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" lgn_status lgn_combine_stats(const lgn_stats_t *parts, int nparts, lgn_stats_t *out) {
+    if (out == nullptr || nparts < 0 || (nparts > 0 && parts == nullptr)) return LGN_ERR_INVALID_ARG;
+    lgn_stats_t t;
+    t.n = 0; t.nnz = 0; t.sum_ln = t.sum_ln2 = t.mu = t.sigma = 0.0;
+    for (int k = 0; k < nparts; ++k) {
+        if (parts[k].nnz > parts[k].n || !std::isfinite(parts[k].sum_ln) || !std::isfinite(parts[k].sum_ln2))
+            return LGN_ERR_INVALID_ARG;
+        t.n += parts[k].n; t.nnz += parts[k].nnz;
+        t.sum_ln += parts[k].sum_ln; t.sum_ln2 += parts[k].sum_ln2;
+    }
+    if (t.nnz) {
+        t.mu = t.sum_ln / (double)t.nnz;
+        double var = t.sum_ln2 / (double)t.nnz - t.mu * t.mu;
+        t.sigma = var > 0.0 ? sqrt(var) : 0.0;
+    }
+    *out = t;
+    return LGN_OK;
+}
+
 extern "C" lgn_status lgn_threshold(double mu, double sigma, double zero_frac, double S, double *tau) {
     if (tau == nullptr) return LGN_ERR_INVALID_ARG;
     *tau = 0.0;
@@ -763,6 +807,61 @@ extern "C" lgn_status lgn_fp_format(double mu, double sigma, int nbits, lgn_fp_f
     if (nbits < 4 || nbits > 8) return LGN_ERR_UNSUPPORTED;
     if (!std::isfinite(mu) || !(sigma >= 0.0) || !std::isfinite(sigma)) return LGN_ERR_INVALID_ARG;
     choose_format(mu, sigma, nbits, *fmt);
+    return LGN_OK;
+}
+
+extern "C" lgn_status lgn_cosine_similarity(double mu, double sigma, double k, double tau, double *cosine) {
+    if (cosine == nullptr) return LGN_ERR_INVALID_ARG;
+    *cosine = 0.0;
+    if (!std::isfinite(mu) || !(sigma >= 0.0) || !std::isfinite(sigma) || !std::isfinite(k)) return LGN_ERR_INVALID_ARG;
+    if (!(tau > 0.0) || !std::isfinite(tau)) return LGN_ERR_INVALID_ARG;
+    const double s = clamp_sigma(sigma), u = log(tau) - mu;
+    if (u > k * s) return LGN_ERR_INVALID_ARG;
+    *cosine = cosine_similarity_of(u, s, k);
+    return LGN_OK;
+}
+
+extern "C" lgn_status lgn_allocate_sparsity(const lgn_alloc_layer_t *layers, int num_layers, int num_deep,
+                                            double S, double s_max, double *S_out, double *achieved) {
+    if (num_layers < 0 || num_deep < 0 || num_deep > num_layers) return LGN_ERR_INVALID_ARG;
+    if (num_layers > 0 && (layers == nullptr || S_out == nullptr)) return LGN_ERR_INVALID_ARG;
+    if (!(S >= 0.0 && S < 1.0) || !(s_max >= S && s_max < 1.0)) return LGN_ERR_INVALID_ARG;
+    double total = 0.0, deep_n = 0.0, deep_zeros = 0.0;
+    for (int i = 0; i < num_layers; ++i) {
+        const lgn_alloc_layer_t &a = layers[i];
+        if (!(a.zero_frac >= 0.0 && a.zero_frac <= 1.0) || !(a.sigma >= 0.0) || !std::isfinite(a.sigma)) return LGN_ERR_INVALID_ARG;
+        if (i < num_deep && (!std::isfinite(a.k) || !(a.min_cos <= 1.0))) return LGN_ERR_INVALID_ARG;
+        total += (double)a.n;
+    }
+    for (int i = 0; i < num_deep; ++i) {
+        const lgn_alloc_layer_t &a = layers[i];
+        const double s = clamp_sigma(a.sigma), l = a.zero_frac;
+        double Si = S;
+        if (l < 1.0 && S > l) {                                   // otherwise nothing is pruned here at S
+            double u = solve_threshold_u(s, (S - l) / (1.0 - l));
+            if (u > a.k * s) u = a.k * s;
+            if (cosine_similarity_of(u, s, a.k) < a.min_cos) {    // below its floor: lower the threshold
+                const double u2 = threshold_u_for_cosine(a.min_cos, s, a.k);
+                double F, dF;
+                pruned_fraction(u2, s, F, dF);
+                Si = l + (1.0 - l) * F;
+                if (Si > S) Si = S;
+            }
+        }
+        S_out[i] = Si;
+        deep_n += (double)a.n;
+        deep_zeros += (double)a.n * Si;
+    }
+    double S_rest = S;
+    const double rest_n = total - deep_n;
+    if (rest_n > 0.0) {
+        S_rest = (S * total - deep_zeros) / rest_n;
+        if (S_rest > s_max) S_rest = s_max;
+        if (S_rest < S) S_rest = S;
+    }
+    double zeros = deep_zeros;
+    for (int i = num_deep; i < num_layers; ++i) { S_out[i] = S_rest; zeros += (double)layers[i].n * S_rest; }
+    if (achieved) *achieved = total > 0.0 ? zeros / total : 0.0;
     return LGN_OK;
 }
 

@@ -98,6 +98,52 @@ LGN_HD double threshold_for(double mu, double sigma, double l, double S) {
     return exp(mu + solve_threshold_u(s, Sp));
 }
 
+// Expected cosine similarity between X and its stochastically pruned copy
+// (appendix "Cosine similarity of stochastic pruning"), for ln X ~ N(mu, s^2) cut
+// off k standard deviations above the mean, at threshold e^(mu+u), u <= k s:
+//     cos^2 = A / B,   A = e^{2 s^2} Phi(k - 2 s)                       (= E[X.T(X)] = E|X|^2)
+//                      B = e^{u + s^2/2} Phi((u - s^2)/s) + A - e^{2 s^2} Phi((u - 2 s^2)/s)
+// Dividing by e^{2 s^2}: B/e^{2s^2} = P + e^{u - 3 s^2/2} Phi((u - s^2)/s) - Phi((u - 2 s^2)/s)
+// with P = Phi(k - 2 s); dB/du = e^{u + s^2/2} Phi((u - s^2)/s) (the two density terms cancel).
+LGN_HD void cosine_terms(double u, double s, double k, double &ratio, double &dratio) {
+    const double P = normal_cdf(k - 2.0 * s);
+    const double g = exp(u - 1.5 * s * s) * normal_cdf((u - s * s) / s);   // also d/du of the bracket
+    const double b = P + g - normal_cdf((u - 2.0 * s * s) / s);
+    ratio = b > 0.0 ? P / b : 1.0;                                          // cos^2
+    dratio = b > 0.0 ? -P * g / (b * b) : 0.0;
+}
+
+LGN_HD double cosine_similarity_of(double u, double s, double k) {
+    double r, dr;
+    cosine_terms(u, s, k, r, dr);
+    return r >= 1.0 ? 1.0 : sqrt(r);
+}
+
+// Largest u <= k s with cosine >= min_cos: Newton on cos^2(u) = min_cos^2 inside a
+// shrinking bracket (cos falls monotonically in u), bisection when a step leaves it.
+LGN_HD double threshold_u_for_cosine(double min_cos, double s, double k) {
+    double hi = k * s, lo = -(40.0 * s + 50.0);
+    if (cosine_similarity_of(hi, s, k) >= min_cos) return hi;
+    const double target = min_cos * min_cos;
+    double u = hi - s;
+    if (!(u > lo)) u = 0.5 * (lo + hi);
+    for (int it = 0; it < 200; ++it) {
+        double r, dr;
+        cosine_terms(u, s, k, r, dr);
+        if (r >= target) lo = u; else hi = u;
+        double un = dr < 0.0 ? u - (r - target) / dr : lo;
+        if (!(un > lo && un < hi)) un = 0.5 * (lo + hi);
+        const double step = fabs(un - u);
+        u = un;
+        if (step <= 4e-16 * fmax(1.0, fabs(u)) || !(hi > lo)) break;
+    }
+    // the answer must satisfy the floor: if rounding put the iterate just past the root,
+    // walk it back by a few units in the last place (doubling), else fall back on the bracket
+    double back = 2.2e-16 * fmax(1.0, fabs(u));
+    for (int j = 0; j < 12 && cosine_similarity_of(u, s, k) < min_cos; ++j, back *= 2.0) u -= back;
+    return cosine_similarity_of(u, s, k) >= min_cos ? u : lo;
+}
+
 LGN_HD float snap_threshold_f32(double tau) {
     float f = (float)tau;                       // round to nearest even
     if (!(f <= FLT_MAX)) f = FLT_MAX;

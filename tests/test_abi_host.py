@@ -189,3 +189,47 @@ def test_scale_from_max(lgn, oracle):
             lgn.lgn_scale_from_max(*bad)
         assert e.value.code == 1
     assert lgn.raw().lgn_scale_from_max(1.0, 4, None) == 1
+
+
+def test_cosine_similarity_agrees_with_oracle(lgn, oracle):
+    for sigma in (0.5, 1.0, 2.0, 3.0, 5.0):
+        for k in (2.0, 2.75, 3.0, 4.0):
+            for mu in (-12.0, 0.0):
+                for u in np.linspace(-6 * sigma, k * sigma, 25):
+                    got = lgn.lgn_cosine_similarity(mu, sigma, k, float(np.exp(mu + u)))
+                    u_eff = float(np.log(np.exp(mu + u)) - mu)            # what the library sees after exp/log
+                    if u_eff > k * sigma:
+                        continue
+                    assert got == pytest.approx(oracle.cosine_similarity(u_eff, sigma, k), rel=1e-11)
+    for bad in [(0.0, 1.0, 3.0, 0.0), (0.0, 1.0, 3.0, -1.0), (0.0, 1.0, 3.0, float("inf")), (float("nan"), 1.0, 3.0, 1.0),
+                (0.0, -1.0, 3.0, 1.0), (0.0, 1.0, 3.0, float(np.exp(3.5)))]:
+        with pytest.raises(lgn.LgnError) as e:
+            lgn.lgn_cosine_similarity(*bad)
+        assert e.value.code == 1
+    assert lgn.raw().lgn_cosine_similarity(0.0, 1.0, 3.0, 1.0, None) == 1
+
+
+def test_allocate_sparsity_agrees_with_oracle(lgn, oracle):
+    rs = np.random.RandomState(3)
+    for trial in range(40):
+        L = int(rs.randint(1, 21))
+        deep = int(rs.randint(0, L + 1))
+        n = [int(x) for x in rs.randint(1_000, 5_000_000, L)]
+        sigma = [float(x) for x in rs.uniform(1.0, 4.0, L)]
+        l = [float(x) for x in rs.uniform(0.0, 0.7, L)]
+        k = [float(x) for x in rs.uniform(2.0, 3.5, L)]
+        floors = [float(x) for x in rs.uniform(0.9, 0.9999, deep)]
+        S, cap = float(rs.choice([0.6, 0.8, 0.9, 0.95])), 0.98
+        want, want_mean = oracle.allocate_sparsity(n, sigma, l, k, floors, S, cap)
+        layers = [dict(n=n[i], sigma=sigma[i], zero_frac=l[i], k=k[i], min_cos=floors[i] if i < deep else 0.0)
+                  for i in range(L)]
+        got, got_mean = lgn.lgn_allocate_sparsity(layers, deep, S, cap)
+        assert got == pytest.approx(want, rel=1e-10, abs=1e-12)
+        assert got_mean == pytest.approx(want_mean, rel=1e-10)
+    with pytest.raises(lgn.LgnError):
+        lgn.lgn_allocate_sparsity([dict(n=1, sigma=1.0, zero_frac=0.0)], 2, 0.5, 0.9)       # more deep layers than layers
+    with pytest.raises(lgn.LgnError):
+        lgn.lgn_allocate_sparsity([dict(n=1, sigma=1.0, zero_frac=0.0)], 0, 0.95, 0.9)      # cap below S
+    with pytest.raises(lgn.LgnError):
+        lgn.lgn_allocate_sparsity([dict(n=1, sigma=1.0, zero_frac=1.5)], 0, 0.5, 0.9)
+    assert lgn.lgn_allocate_sparsity([], 0, 0.5, 0.9) == ([], 0.0)

@@ -77,3 +77,57 @@ def test_bench_workload_full_size(lgn, oracle):
             ref = oracle.prune(np_bits(g[lo:hi]), tau, 1000 + k, first=lo)
             got = np_bits(o[lo:hi])
             assert np.array_equal(got.view(np.uint32), ref.view(np.uint32)), (k, lo)
+
+
+@pytest.mark.parametrize("mode", ["quant", "prune"])
+def test_bf16_group_with_large_queue_items(lgn, oracle, mode):
+    """A bf16 group large enough (1.4 GB of input) for the library to hand out two
+    sub-tiles per queue item: ResNet-50 shapes at batch 64, one grouped call.  Every
+    layer's statistics against the oracle; codes / pruned values bit for bit on windows
+    that straddle item and tile boundaries, and on the smallest layers in full."""
+    name = "resnet50_bs256_bf16_fp6" if mode == "quant" else "resnet50_bs256_bf16_prune"
+    w, specs = bench.workload_specs(name, 64, 0)
+    tensors = synth.make_layers(specs, torch.bfloat16, "cuda")
+    assert sum(t.numel() for t in tensors) * 2 > 8 * 592 * (128 << 10)
+    dev = tensors[0].device
+    ref_stats = [oracle.stats(np_bits(g)) for g in tensors]
+    if mode == "quant":
+        outs = [torch.empty(lgn.lgn_codes_bytes(g.numel(), 6) + 16, dtype=torch.uint8, device=dev) for g in tensors]
+        layers = [lgn.make_layer(g, o, lgn.MODE_QUANTIZE, nbits=6, rounding=lgn.ROUND_STOCHASTIC, seed=500 + k,
+                                 mu_override=st["mu"], sigma_override=st["sigma"])
+                  for k, (g, o, st) in enumerate(zip(tensors, outs, ref_stats))]
+    else:
+        outs = [torch.empty_like(g) for g in tensors]
+        layers = [lgn.make_layer(g, o, lgn.MODE_PRUNE, S=s.sparsity, seed=500 + k,
+                                 mu_override=st["mu"], sigma_override=st["sigma"])
+                  for k, (g, o, s, st) in enumerate(zip(tensors, outs, specs, ref_stats))]
+    ws = lgn.new_workspace([g.numel() for g in tensors], dev)
+    res = lgn.new_results(len(tensors), dev)
+    lgn.lgn_compress_layers(layers, res, ws)
+    torch.cuda.synchronize()
+    results = lgn.read_results(res, len(tensors))
+    rs = np.random.RandomState(1)
+    for k, (g, o, r, s, st) in enumerate(zip(tensors, outs, results, specs, ref_stats)):
+        assert r["status"] == 0
+        assert_stats_close(r, st)
+        n = g.numel()
+        if n <= 2_000_000:
+            windows = [(0, n)]
+        else:
+            starts = [0, 65536 - 4096, 2 * 65536 - 4096, n - 8192] + [int(x) // 8 * 8 for x in rs.randint(0, n - 8192, 2)]
+            windows = [(a, a + 8192) for a in starts]
+        if mode == "quant":
+            fmt = oracle.fp_format(st["mu"], st["sigma"], st["nnz"], 6)
+            assert r["fmt"] == fmt
+            got_all = o.cpu().numpy()
+            for lo, hi in windows:                        # windows start on multiples of 8 elements = 6 bytes
+                codes = oracle.quantize(np_bits(g[lo:hi]), fmt["exp_bits"], fmt["man_bits"], fmt["scale_exp"], 1, 500 + k, first=lo)
+                ref = oracle.pack(codes, 6)
+                nbytes = (hi - lo) * 6 // 8
+                assert np.array_equal(got_all[lo * 6 // 8: lo * 6 // 8 + nbytes], ref[:nbytes]), (k, lo)
+        else:
+            tau = oracle.snap_tau(oracle.threshold(st["mu"], st["sigma"], st["zero_frac"], s.sparsity), oracle.BF16) if st["nnz"] else 0.0
+            assert r["tau"] == tau
+            for lo, hi in windows:
+                ref = oracle.prune(np_bits(g[lo:hi]), tau, 500 + k, first=lo)
+                assert np.array_equal(np_bits(o[lo:hi]), ref), (k, lo)
