@@ -150,18 +150,18 @@ __device__ __forceinline__ void st_release(uint32_t *p, uint32_t v) {
 // The out-of-line statistics tile: ragged last tiles, and the extended form (a
 // right-mode mask and / or max|g|).  Does the whole item: the tile, the CTA
 // reduction (one barrier) and the partial.
-template <int DT>
+template <int DT, int TILE>
 __device__ __noinline__ void run_stats_tile_slow(const LayerState &L, uint32_t tile, bool ext, Partial *partials, double *sm);
 
 // One tile's sums: per-warp shuffle tree, eight warp results through shared
 // memory, added in warp order by thread 0, which also stores the tile's partial.
 // One barrier; `sm` is reused only after the caller's next barrier.
-template <int DT, bool INLINE_HOT>
+template <int DT, bool INLINE_HOT, int TILE>
 __device__ __forceinline__ void run_stats_tile(const LayerState &L, uint32_t tile, bool ext, Partial *partials, double *sm) {
-    const uint64_t base = (uint64_t)tile * kTileElems;
-    if (!INLINE_HOT || ext || base + kTileElems > L.n) { run_stats_tile_slow<DT>(L, tile, ext, partials, sm); return; }
+    const uint64_t base = (uint64_t)tile * TILE;
+    if (!INLINE_HOT || ext || base + TILE > L.n) { run_stats_tile_slow<DT, TILE>(L, tile, ext, partials, sm); return; }
     StatsAcc acc;
-    stats_tile<DT, true>(L.g, base, L.n, acc);
+    stats_tile<DT, true, TILE>(L.g, base, L.n, acc);
     #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
         acc.s1 += __shfl_down_sync(0xFFFFFFFFu, acc.s1, off);
@@ -185,13 +185,13 @@ __device__ __forceinline__ void run_stats_tile(const LayerState &L, uint32_t til
     }
 }
 
-template <int DT>
+template <int DT, int TILE>
 __device__ __noinline__ void run_stats_tile_slow(const LayerState &L, uint32_t tile, bool ext, Partial *partials, double *sm) {
     StatsAcc acc;
-    const uint64_t base = (uint64_t)tile * kTileElems;
-    if (!ext)        stats_tile<DT, false>(L.g, base, L.n, acc);
-    else if (L.mask) stats_tile_ext<DT, true>(L.g, L.mask, base, L.n, acc);
-    else             stats_tile_ext<DT, false>(L.g, nullptr, base, L.n, acc);
+    const uint64_t base = (uint64_t)tile * TILE;
+    if (!ext)        stats_tile<DT, false, TILE>(L.g, base, L.n, acc);
+    else if (L.mask) stats_tile_ext<DT, true, TILE>(L.g, L.mask, base, L.n, acc);
+    else             stats_tile_ext<DT, false, TILE>(L.g, nullptr, base, L.n, acc);
     warp_reduce(acc, 32);
     const int w = threadIdx.x >> 5;
     if ((threadIdx.x & 31) == 0) {
@@ -213,38 +213,38 @@ __device__ __noinline__ void run_stats_tile_slow(const LayerState &L, uint32_t t
     }
 }
 
-template <int DT>
+template <int DT, int TILE>
 __device__ __noinline__ void prune_tile_general(const void *g, void *out, uint64_t base, uint64_t n,
                                                 float tau, uint64_t seed, const Weyl &wy) {
-    prune_tile<DT, false>(g, out, base, n, tau, seed, wy);
+    prune_tile<DT, false, TILE>(g, out, base, n, tau, seed, wy);
 }
 
-template <int DT, bool INLINE_HOT>
+template <int DT, bool INLINE_HOT, int TILE>
 __device__ __forceinline__ void run_prune_tile(const void *g, void *out, uint64_t n, uint32_t tile,
                                                float tau, uint64_t seed, const Weyl &wy) {
-    const uint64_t base = (uint64_t)tile * kTileElems;
+    const uint64_t base = (uint64_t)tile * TILE;
     const bool tiny = tau > 0.f && tau < kPruneFastMin;       // alpha*2^-16 inexact, or alpha*eps could round to zero
-    if (INLINE_HOT && base + kTileElems <= n && !tiny) prune_tile<DT, true>(g, out, base, n, tau, seed, wy);
-    else                                               prune_tile_general<DT>(g, out, base, n, tau, seed, wy);
+    if (INLINE_HOT && base + TILE <= n && !tiny) prune_tile<DT, true, TILE>(g, out, base, n, tau, seed, wy);
+    else                                         prune_tile_general<DT, TILE>(g, out, base, n, tau, seed, wy);
 }
 
-template <int DT, int NBITS, bool SR>
+template <int DT, int NBITS, bool SR, int TILE>
 __device__ __noinline__ void quant_tile_general(const void *g, uint32_t *codes, uint64_t base, uint64_t n,
                                                 uint64_t total_words, const QuantParams &q, uint64_t seed,
                                                 const Weyl &wy) {
-    quant_tile<DT, NBITS, SR, false, false>(g, codes, base, n, total_words, q, seed, wy);
+    quant_tile<DT, NBITS, SR, false, false, TILE>(g, codes, base, n, total_words, q, seed, wy);
 }
 
-template <int DT, int NBITS, bool SR, bool INLINE_HOT>
+template <int DT, int NBITS, bool SR, bool INLINE_HOT, int TILE>
 __device__ __forceinline__ void run_quant_tile(const void *g, void *out, uint64_t n, uint32_t tile,
                                                const QuantParams &q, uint64_t seed, const Weyl &wy) {
-    const uint64_t base = (uint64_t)tile * kTileElems;
+    const uint64_t base = (uint64_t)tile * TILE;
     const uint64_t total_words = (n * (uint64_t)NBITS + 31) >> 5;
     uint32_t *codes = static_cast<uint32_t *>(out);
-    if (INLINE_HOT && base + kTileElems <= n && q.K >= 1 && q.K <= 255)
-        quant_tile<DT, NBITS, SR, true, true>(g, codes, base, n, total_words, q, seed, wy);
+    if (INLINE_HOT && base + TILE <= n && q.K >= 1 && q.K <= 255)
+        quant_tile<DT, NBITS, SR, true, true, TILE>(g, codes, base, n, total_words, q, seed, wy);
     else
-        quant_tile_general<DT, NBITS, SR>(g, codes, base, n, total_words, q, seed, wy);
+        quant_tile_general<DT, NBITS, SR, TILE>(g, codes, base, n, total_words, q, seed, wy);
 }
 
 // run-time dispatch for groups whose layers differ in type, mode or width
@@ -252,8 +252,8 @@ template <int DT>
 __device__ __forceinline__ void run_quant_tile_any(const void *g, void *out, uint64_t n, uint32_t tile, int nbits,
                                                    const QuantParams &q, bool sr, uint64_t seed, const Weyl &wy) {
     #define LGN_Q(NB) \
-        if (sr) run_quant_tile<DT, NB, true, false>(g, out, n, tile, q, seed, wy); \
-        else    run_quant_tile<DT, NB, false, false>(g, out, n, tile, q, seed, wy);
+        if (sr) run_quant_tile<DT, NB, true, false, kTileElems>(g, out, n, tile, q, seed, wy); \
+        else    run_quant_tile<DT, NB, false, false, kTileElems>(g, out, n, tile, q, seed, wy);
     switch (nbits) {
         case 4: LGN_Q(4) break;
         case 5: LGN_Q(5) break;
@@ -358,7 +358,7 @@ constexpr int kAny = -1;                      // template value: decided per lay
 // layers may ask for the extended statistics tile (a right-mode mask, max|g|);
 // every specialised kernel exists without and (as a second instance) with it, so a
 // group that does not ask pays nothing for it.
-template <int DT, int MODE, int NBITS, int SR, bool EXT = false>
+template <int DT, int MODE, int NBITS, int SR, bool EXT = false, int TILE = kTileElems>
 __global__ void __launch_bounds__(kThreads, kMinCtas)
 compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Segment *segs,
                 int num_layers, uint32_t total_items, Partial *partials) {
@@ -416,10 +416,10 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
         if (sg.phase != kPhaseApply) {
             const bool ext = (EXT || !kSpecial) && sg.phase == kPhaseStatsExt;
             if constexpr (kSpecial) {
-                run_stats_tile<DT, true>(L, tile, ext, partials, sm_red);
+                run_stats_tile<DT, true, TILE>(L, tile, ext, partials, sm_red);
             } else {
-                if (L.dt == LGN_BF16) run_stats_tile<LGN_BF16, false>(L, tile, ext, partials, sm_red);
-                else                  run_stats_tile<LGN_F32, false>(L, tile, ext, partials, sm_red);
+                if (L.dt == LGN_BF16) run_stats_tile<LGN_BF16, false, kTileElems>(L, tile, ext, partials, sm_red);
+                else                  run_stats_tile<LGN_F32, false, kTileElems>(L, tile, ext, partials, sm_red);
             }
             if (threadIdx.x == 0) {
                 __threadfence();                                   // the partial before the ticket
@@ -445,15 +445,15 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
                 ready_layer = (int)sg.layer;
             }
             if constexpr (kSpecial && MODE == LGN_MODE_PRUNE) {
-                run_prune_tile<DT, true>(L.g, L.out, L.n, tile, __ldcg(&D->tau), L.seed, wy);
+                run_prune_tile<DT, true, TILE>(L.g, L.out, L.n, tile, __ldcg(&D->tau), L.seed, wy);
             } else if constexpr (kSpecial && MODE == LGN_MODE_QUANTIZE) {
                 const QuantParams q = load_quant_params(D);
-                run_quant_tile<DT, NBITS, SR != 0, true>(L.g, L.out, L.n, tile, q, L.seed, wy);
+                run_quant_tile<DT, NBITS, SR != 0, true, TILE>(L.g, L.out, L.n, tile, q, L.seed, wy);
             } else if constexpr (!kSpecial) {
                 if (L.mode == LGN_MODE_PRUNE) {
                     const float tau = __ldcg(&D->tau);
-                    if (L.dt == LGN_BF16) run_prune_tile<LGN_BF16, false>(L.g, L.out, L.n, tile, tau, L.seed, wy);
-                    else                  run_prune_tile<LGN_F32, false>(L.g, L.out, L.n, tile, tau, L.seed, wy);
+                    if (L.dt == LGN_BF16) run_prune_tile<LGN_BF16, false, kTileElems>(L.g, L.out, L.n, tile, tau, L.seed, wy);
+                    else                  run_prune_tile<LGN_F32, false, kTileElems>(L.g, L.out, L.n, tile, tau, L.seed, wy);
                 } else {
                     const QuantParams q = load_quant_params(D);
                     const bool sr = L.rounding == LGN_ROUND_STOCHASTIC;
@@ -470,7 +470,7 @@ template <int DT>
 __global__ void __launch_bounds__(kThreads, kMinCtas)
 prune_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, float tau, uint64_t seed, Weyl wy) {
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)
-        run_prune_tile<DT, true>(g, out, n, tile, tau, seed, wy);
+        run_prune_tile<DT, true, kTileElems>(g, out, n, tile, tau, seed, wy);
 }
 
 template <int DT, int NBITS, int SR>
@@ -478,7 +478,7 @@ __global__ void __launch_bounds__(kThreads, kMinCtas)
 quantize_kernel(const void *g, void *out, uint64_t n, uint32_t ntiles, const __grid_constant__ QuantParams q,
                 uint64_t seed, Weyl wy) {
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x)
-        run_quant_tile<DT, NBITS, SR != 0, true>(g, out, n, tile, q, seed, wy);
+        run_quant_tile<DT, NBITS, SR != 0, true, kTileElems>(g, out, n, tile, q, seed, wy);
 }
 
 // ------------------------------------------------------------------ kernel tables
@@ -501,6 +501,19 @@ constexpr int kVariantPruneExt = 12, kVariantQuantExt0 = 13;
     LGN_CKX(DT, LGN_MODE_QUANTIZE, 7, 0), LGN_CKX(DT, LGN_MODE_QUANTIZE, 7, 1), \
     LGN_CKX(DT, LGN_MODE_QUANTIZE, 8, 0), LGN_CKX(DT, LGN_MODE_QUANTIZE, 8, 1) }
 static const void *const kCompressTable[2][kVariants] = { LGN_CK_ROW(LGN_F32), LGN_CK_ROW(LGN_BF16) };
+// bf16 with tiles of twice the elements (the same 128 KiB of input per tile as fp32): large calls only
+constexpr int kBigTileElems = 2 * kTileElems;
+#define LGN_CKB(MODE, NB, SR, EXT) reinterpret_cast<const void *>(&compress_kernel<LGN_BF16, MODE, NB, SR, EXT, kBigTileElems>)
+#define LGN_CKB_ROW(EXT) LGN_CKB(LGN_MODE_QUANTIZE, 4, 0, EXT), LGN_CKB(LGN_MODE_QUANTIZE, 4, 1, EXT), \
+    LGN_CKB(LGN_MODE_QUANTIZE, 5, 0, EXT), LGN_CKB(LGN_MODE_QUANTIZE, 5, 1, EXT), \
+    LGN_CKB(LGN_MODE_QUANTIZE, 6, 0, EXT), LGN_CKB(LGN_MODE_QUANTIZE, 6, 1, EXT), \
+    LGN_CKB(LGN_MODE_QUANTIZE, 7, 0, EXT), LGN_CKB(LGN_MODE_QUANTIZE, 7, 1, EXT), \
+    LGN_CKB(LGN_MODE_QUANTIZE, 8, 0, EXT), LGN_CKB(LGN_MODE_QUANTIZE, 8, 1, EXT)
+static const void *const kCompressTableBig[kVariants] = {
+    LGN_CKB(kModeStatsOnly, kAny, kAny, false), LGN_CKB(LGN_MODE_PRUNE, kAny, kAny, false), LGN_CKB_ROW(false),
+    LGN_CKB(LGN_MODE_PRUNE, kAny, kAny, true), LGN_CKB_ROW(true) };
+#undef LGN_CKB_ROW
+#undef LGN_CKB
 static const void *const kCompressGeneral = LGN_CK(kAny, kAny, kAny, kAny);
 #undef LGN_CK_ROW
 #undef LGN_CK
@@ -669,10 +682,24 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
     int grid = persistent_ctas(fn);
     if (grid < 1) return LGN_ERR_CUDA;
 
+    // Tile size.  128 KiB of input per tile is the measured optimum for both types: 32768 fp32
+    // or 65536 bf16 elements.  The larger bf16 tile is used only when the call has enough of
+    // them (eight rounds of the grid) for the coarser tail of the queue not to matter.
+    uint32_t tile_elems = kTileElems;
+    if (fn != kCompressGeneral && st[0].dt == LGN_BF16 && !withhold_tile) {
+        uint64_t big_tiles = 0;
+        for (int k = 0; k < L; ++k) big_tiles += st[k].n / kBigTileElems;
+        if (big_tiles >= 8ull * (uint64_t)grid) {
+            for (int v = 0; v < kVariants; ++v)
+                if (kCompressTable[LGN_BF16][v] == fn) { fn = kCompressTableBig[v]; tile_elems = kBigTileElems; break; }
+            grid = persistent_ctas(fn);
+            if (grid < 1) return LGN_ERR_CUDA;
+        }
+    }
     uint32_t partial0 = 0;
     for (int k = 0; k < L; ++k) {
         LayerState &s = st[k];
-        s.ntiles = (uint32_t)((s.n + kTileElems - 1) / kTileElems);
+        s.ntiles = (uint32_t)((s.n + tile_elems - 1) / tile_elems);
         s.partial0 = partial0;
         partial0 += s.ntiles;
     }

@@ -245,10 +245,10 @@ struct StatsAcc {            // per thread, in log2 units
 // variance of exactly zero.  Runs go to fp64 accumulators; the pivot is taken
 // out again in fp64 at the end of the tile:
 //   sum y = sum d + c P,   sum y^2 = sum d^2 + 2 P sum d + c P^2.
-template <int DT, bool FULL>
+template <int DT, bool FULL, int TILE = kTileElems>
 __device__ __forceinline__ void stats_tile(const void *g, uint64_t tile_base, uint64_t n, StatsAcc &acc) {
     constexpr int C = ElemTraits<DT>::kChunk;
-    constexpr int kLoads = kTileElems / (kThreads * C);   // 8 (fp32) or 4 (bf16)
+    constexpr int kLoads = TILE / (kThreads * C);   // 8 (fp32) or 4 (bf16)
     constexpr int kGroup = 16 / C;                        // chunks per register buffer (two buffers): one run of 16
     const float kUnset = -__int_as_float(0x7F800000);     // -inf: no nonzero seen yet
     float P = kUnset;
@@ -311,11 +311,11 @@ __device__ __forceinline__ void load_mask_chunk(const uint8_t *mask, uint64_t i,
     }
 }
 
-template <int DT, bool MASKED>
+template <int DT, bool MASKED, int TILE = kTileElems>
 __device__ __forceinline__ void stats_tile_ext(const void *g, const uint8_t *mask, uint64_t tile_base, uint64_t n,
                                                StatsAcc &acc) {
     constexpr int C = ElemTraits<DT>::kChunk;
-    constexpr int kLoads = kTileElems / (kThreads * C);
+    constexpr int kLoads = TILE / (kThreads * C);
     const float kUnset = -__int_as_float(0x7F800000);
     float P = kUnset, amax = 0.f;
     double D1 = 0.0, D2 = 0.0;
@@ -449,11 +449,11 @@ __device__ __forceinline__ uint32_t prune_pair_bf16(uint32_t w, uint32_t r, floa
 }
 
 // tau == 0 never reaches the fast forms' arithmetic (the tile is copied instead).
-template <int DT, bool FULL>
+template <int DT, bool FULL, int TILE = kTileElems>
 __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t tile_base, uint64_t n,
                                            float tau, uint64_t seed, const Weyl &wy) {
     constexpr int C = ElemTraits<DT>::kChunk;
-    constexpr int kLoads = kTileElems / (kThreads * C);
+    constexpr int kLoads = TILE / (kThreads * C);
     constexpr int kGroup = 1;                             // one chunk per buffer: the apply bodies need the registers
     constexpr bool ZCHECK = !FULL;                        // the general body also serves tiny thresholds
     const float c = tau * 0x1p-16f;                       // used by the hot path only (FULL: alpha >= kPruneFastMin or 0)
@@ -655,13 +655,13 @@ __device__ __forceinline__ uint32_t quant_pair_bf16(uint32_t w, uint32_t r, cons
 // not a multiple of 32, the first bits of the next lane (one warp shuffle), so
 // every store is an aligned 32-bit word of the little-endian bit stream.
 // `total_words` = words in the whole stream.
-template <int DT, int NBITS, bool SR, bool FAST, bool FULL>
+template <int DT, int NBITS, bool SR, bool FAST, bool FULL, int TILE = kTileElems>
 __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint64_t tile_base, uint64_t n,
                                            uint64_t total_words, const QuantParams &q, uint64_t seed, const Weyl &wy) {
     constexpr int C = ElemTraits<DT>::kChunk;
     constexpr int B = C * NBITS;                           // bits per lane per load step: 32..128
     constexpr int NW = (B + 31) / 32;                      // words that hold a lane's bits
-    constexpr int kLoads = kTileElems / (kThreads * C);
+    constexpr int kLoads = TILE / (kThreads * C);
     constexpr int kGroup = 1;
     const int lane = threadIdx.x & 31;
     const int o0 = (B % 32 == 0) ? 0 : ((32 - ((lane * B) & 31)) & 31);   // first word boundary inside this lane
