@@ -70,6 +70,8 @@ for _lg in (26, 28):
                                                          dtype="f32" if _dt == "fp32" else "bf16", mode="quant")
         WORKLOADS[f"quantile_{_dt}_2p{_lg}"] = dict(net="aux", kind="quantile", log2n=_lg,
                                                     dtype="f32" if _dt == "fp32" else "bf16", mode="quantile")
+        WORKLOADS[f"prefix_decode_{_dt}_2p{_lg}"] = dict(net="aux", kind="prefix", decode=True, log2n=_lg,
+                                                         dtype="f32" if _dt == "fp32" else "bf16", mode="prefix")
         WORKLOADS[f"prefix_encode_{_dt}_2p{_lg}"] = dict(net="aux", kind="prefix", log2n=_lg,
                                                          dtype="f32" if _dt == "fp32" else "bf16", mode="prefix")
 
@@ -403,6 +405,11 @@ def run_aux(args):
         alg_bytes = n * esize + 4.0 * words          # one read of the tensor + the stream written
         kernel = "prefix_encode_kernel"
         launches = 1
+        if w.get("decode"):                          # the inverse: the stream read + the tensor written
+            dec_out = torch.empty_like(g)
+            sd = stream_dev[:words]
+            call = lambda: lgn.lgn_prefix_decode(sd, off_dev, dec_out, tau)
+            kernel = "prefix_decode_kernel"
     for _ in range(args.warmup):
         call()
     torch.cuda.synchronize()

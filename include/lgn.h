@@ -22,7 +22,7 @@
  *  - Tensors are contiguous and are treated as flat arrays of n elements; the
  *    element index used for randomness is the flat index.
  *  - Gradient tensors (g, and out of a pruning call) must be 32-byte aligned;
- *    code streams, workspaces and result arrays 16-byte aligned.  Input and
+ *    code streams and workspaces 16-byte aligned, result arrays 8-byte aligned.  Input and
  *    output buffers must not overlap.
  *  - Inputs must be finite, with magnitudes below 2^104 (about 2e31).  +0 and -0
  *    both count as zero.
@@ -382,7 +382,11 @@ lgn_status lgn_stats_static_scratch(const void *g, uint64_t n, lgn_dtype dt, lgn
 
 /* The grouped path for tensors that live in HOST memory: copies every input to
  * the device, runs lgn_compress_layers, copies every output and the results
- * back, and waits for the stream.  This is the end-to-end form of the call a
+ * back, and waits until all of it has landed.  The layers go through in groups of
+ * consecutive layers (about 64 MB of input each) on three streams (the caller's for
+ * the kernels, two that the call creates and destroys for the copies), so that
+ * copies in, kernels and copies out of neighbouring groups overlap; each layer's
+ * output and result are those of the single grouped call.  This is the end-to-end form of the call a
  * training loop on another device (or a test harness) makes; the paper's own
  * setting keeps the gradients on the accelerator and needs no copy.
  *   layers        host array; g and out of each entry are HOST pointers
@@ -391,7 +395,7 @@ lgn_status lgn_stats_static_scratch(const void *g, uint64_t n, lgn_dtype dt, lgn
  *   dev_buf       device scratch of at least lgn_host_staging_bytes(layers,
  *                 num_layers) bytes, 256-byte aligned; holds the device copies
  *                 of inputs and outputs, the results and the workspace
- * Returns after cudaStreamSynchronize(stream). */
+ * Returns after the three streams have drained. */
 size_t lgn_host_staging_bytes(const lgn_layer_t *layers, int num_layers);
 lgn_status lgn_compress_layers_host(const lgn_layer_t *layers, int num_layers,
                                     lgn_layer_result_t *results_host,

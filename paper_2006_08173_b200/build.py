@@ -10,7 +10,8 @@ _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "liblgn.so")
 SOURCES = [os.path.join(_CSRC, "lgn.cu"), os.path.join(_CSRC, "lgn_prefix.cu"),
-           os.path.join(_CSRC, "lgn_dequant.cu"), os.path.join(_CSRC, "lgn_quantile.cu")]
+           os.path.join(_CSRC, "lgn_dequant.cu"), os.path.join(_CSRC, "lgn_quantile.cu"),
+           os.path.join(_CSRC, "lgn_host.cu")]
 _DEPS = SOURCES + [os.path.join(_CSRC, "lgn_device.cuh"), os.path.join(_CSRC, "lgn_closed_form.cuh"),
                    os.path.join(_ROOT, "include", "lgn.h")]
 

@@ -535,6 +535,7 @@ static int variant_of(int mode, int nbits, int rounding) {
 }
 
 // ------------------------------------------------------------------ host side
+static bool aligned8(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 7u) == 0; }
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static bool aligned32(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
 
@@ -964,7 +965,7 @@ extern "C" lgn_status lgn_compress_layers(const lgn_layer_t *layers, int num_lay
                                           void *ws, size_t ws_bytes, void *stream) {
     if (num_layers < 0) return LGN_ERR_INVALID_ARG;
     if (num_layers == 0) return LGN_OK;
-    if (layers == nullptr || results_dev == nullptr || !aligned16(results_dev)) return LGN_ERR_INVALID_ARG;
+    if (layers == nullptr || results_dev == nullptr || !aligned8(results_dev)) return LGN_ERR_INVALID_ARG;
     std::vector<InternalLayer> v((size_t)num_layers);
     for (int k = 0; k < num_layers; ++k) {
         if (layers[k].mode != LGN_MODE_PRUNE && layers[k].mode != LGN_MODE_QUANTIZE) return LGN_ERR_INVALID_ARG;
@@ -975,42 +976,10 @@ extern "C" lgn_status lgn_compress_layers(const lgn_layer_t *layers, int num_lay
     return run_layers(v, ws, ws_bytes, static_cast<cudaStream_t>(stream));
 }
 
-// ------------------------------------------------------------------ host-buffer form
-namespace {
-struct StagingPlan {
-    std::vector<size_t> in_off, out_off, mask_off, in_bytes, out_bytes;
-    size_t results_off = 0, ws_off = 0, ws_bytes = 0, total = 0;
-};
-
-bool plan_staging(const lgn_layer_t *layers, int L, StagingPlan &p) {
-    size_t off = 0;
-    std::vector<uint64_t> ns((size_t)L);
-    p.in_off.resize(L); p.out_off.resize(L); p.mask_off.resize(L); p.in_bytes.resize(L); p.out_bytes.resize(L);
-    for (int k = 0; k < L; ++k) {
-        const lgn_layer_t &d = layers[k];
-        if (d.dt != LGN_F32 && d.dt != LGN_BF16) return false;
-        if (d.mode == LGN_MODE_QUANTIZE && (d.nbits < 4 || d.nbits > 8)) return false;
-        if (d.mode != LGN_MODE_QUANTIZE && d.mode != LGN_MODE_PRUNE) return false;
-        ns[k] = d.n;
-        p.in_bytes[k] = (size_t)d.n * (d.dt == LGN_BF16 ? 2u : 4u);
-        p.out_bytes[k] = d.mode == LGN_MODE_PRUNE ? p.in_bytes[k] : lgn_codes_bytes(d.n, d.nbits);
-        p.in_off[k] = off;  off += round_up(p.in_bytes[k], 256);
-        p.out_off[k] = off; off += round_up(p.out_bytes[k], 256);
-        p.mask_off[k] = off; if (d.right_mode) off += round_up((size_t)d.n, 256);
-    }
-    p.results_off = off; off += round_up(sizeof(lgn_layer_result_t) * (size_t)L, 256);
-    WsLayout w;
-    if (!ws_layout(ns.data(), L, w)) return false;
-    p.ws_off = off; p.ws_bytes = w.total; off += w.total;
-    p.total = off;
-    return true;
-}
-}  // namespace
-
 extern "C" lgn_status lgn_selftest_wait_expires(const lgn_layer_t *layers, int num_layers,
                                                 lgn_layer_result_t *results_dev,
                                                 void *ws, size_t ws_bytes, void *stream) {
-    if (num_layers <= 0 || layers == nullptr || results_dev == nullptr || !aligned16(results_dev))
+    if (num_layers <= 0 || layers == nullptr || results_dev == nullptr || !aligned8(results_dev))
         return LGN_ERR_INVALID_ARG;
     std::vector<InternalLayer> v((size_t)num_layers);
     for (int k = 0; k < num_layers; ++k) {
@@ -1021,54 +990,6 @@ extern "C" lgn_status lgn_selftest_wait_expires(const lgn_layer_t *layers, int n
     }
     if (layers[0].n == 0) return LGN_ERR_INVALID_ARG;
     return run_layers(v, ws, ws_bytes, static_cast<cudaStream_t>(stream), true);
-}
-
-extern "C" size_t lgn_host_staging_bytes(const lgn_layer_t *layers, int num_layers) {
-    if (num_layers <= 0 || layers == nullptr) return 0;
-    StagingPlan p;
-    return plan_staging(layers, num_layers, p) ? p.total : 0;
-}
-
-extern "C" lgn_status lgn_compress_layers_host(const lgn_layer_t *layers, int num_layers,
-                                               lgn_layer_result_t *results_host,
-                                               void *dev_buf, size_t dev_bytes, void *stream) {
-    if (num_layers < 0) return LGN_ERR_INVALID_ARG;
-    if (num_layers == 0) return LGN_OK;
-    if (layers == nullptr || results_host == nullptr || dev_buf == nullptr) return LGN_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(dev_buf) & 255u) != 0) return LGN_ERR_INVALID_ARG;
-    StagingPlan p;
-    if (!plan_staging(layers, num_layers, p)) return LGN_ERR_INVALID_ARG;
-    if (dev_bytes < p.total) return LGN_ERR_WORKSPACE;
-    for (int k = 0; k < num_layers; ++k)
-        if (layers[k].n > 0 && (layers[k].g == nullptr || layers[k].out == nullptr)) return LGN_ERR_INVALID_ARG;
-
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    char *base = static_cast<char *>(dev_buf);
-    std::vector<lgn_layer_t> dev_layers(layers, layers + num_layers);
-    for (int k = 0; k < num_layers; ++k) {
-        dev_layers[k].g = base + p.in_off[k];
-        dev_layers[k].out = base + p.out_off[k];
-        if (p.in_bytes[k] &&
-            cudaMemcpyAsync(base + p.in_off[k], layers[k].g, p.in_bytes[k], cudaMemcpyHostToDevice, st) != cudaSuccess)
-            return LGN_ERR_CUDA;
-        if (layers[k].right_mode) {
-            dev_layers[k].right_mode = base + p.mask_off[k];
-            if (layers[k].n &&
-                cudaMemcpyAsync(base + p.mask_off[k], layers[k].right_mode, (size_t)layers[k].n, cudaMemcpyHostToDevice, st) != cudaSuccess)
-                return LGN_ERR_CUDA;
-        }
-    }
-    lgn_layer_result_t *res_dev = reinterpret_cast<lgn_layer_result_t *>(base + p.results_off);
-    lgn_status s = lgn_compress_layers(dev_layers.data(), num_layers, res_dev, base + p.ws_off, p.ws_bytes, stream);
-    if (s != LGN_OK) { cudaStreamSynchronize(st); return s; }
-    for (int k = 0; k < num_layers; ++k)
-        if (p.out_bytes[k] &&
-            cudaMemcpyAsync(layers[k].out, base + p.out_off[k], p.out_bytes[k], cudaMemcpyDeviceToHost, st) != cudaSuccess)
-            return LGN_ERR_CUDA;
-    if (cudaMemcpyAsync(results_host, res_dev, sizeof(lgn_layer_result_t) * (size_t)num_layers,
-                        cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return LGN_ERR_CUDA;
-    return cudaStreamSynchronize(st) == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
 }
 
 // ------------------------------------------------------------------ statistics without a caller workspace

@@ -264,40 +264,65 @@ prefix_encode_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host
 
 __global__ void prefix_empty_kernel(uint64_t *off) { off[0] = 0ull; }
 
-// One thread decodes one block.
+// One thread decodes one block (the code is sequential within a block); a warp takes 32
+// consecutive blocks.  Every lane decodes 32 elements of its block into a row of a
+// shared-memory tile, then the warp writes the 32 rows out, one coalesced store per row,
+// so that the output leaves in whole 128-byte (fp32) or 64-byte (bf16) pieces.  The next
+// stream word of a lane is loaded one refill ahead of its use.
+constexpr int kDecThreads = 128;
 template <int DT>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kDecThreads)
 prefix_decode_kernel(const uint32_t *stream, const uint64_t *off, uint64_t n, uint64_t nblocks, float tau_host,
                      const lgn_layer_result_t *tau_from, void *out) {
-    const uint64_t b = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (b >= nblocks) return;
+    __shared__ uint32_t tile[kDecThreads / 32][32][33];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint64_t b0 = ((uint64_t)blockIdx.x * kDecThreads + threadIdx.x) & ~31ull;   // first block of this warp
+    const uint64_t b = b0 + lane;
+    if (b0 >= nblocks) return;                                   // whole warp
     const uint32_t tp = tau_pattern<DT>(pfx_tau(tau_host, tau_from));
-    const uint32_t *p = stream + off[b], *end = stream + off[b + 1];
+    const bool live = b < nblocks;
+    const uint32_t *p = stream, *end = stream;
+    if (live) { p = stream + off[b]; end = stream + off[b + 1]; }
     unsigned long long buf = 0ull;
     int have = 0;
+    uint32_t ahead = p < end ? *p : 0u;                          // the word at p, already on its way
     const uint64_t i0 = b * LGN_PREFIX_BLOCK;
-    const uint64_t i1 = i0 + LGN_PREFIX_BLOCK < n ? i0 + LGN_PREFIX_BLOCK : n;
+    const uint64_t i1 = !live ? i0 : (i0 + LGN_PREFIX_BLOCK < n ? i0 + LGN_PREFIX_BLOCK : n);
     auto refill = [&]() {                                        // keeps 33..64 bits in hand (zeros past the block)
         if (have <= 32) {
-            const unsigned long long w = p < end ? *p : 0u;
-            ++p;
-            buf |= w << have;
+            buf |= (unsigned long long)ahead << have;
             have += 32;
+            ++p;
+            ahead = p < end ? *p : 0u;
         }
     };
-    for (uint64_t i = i0; i < i1; ++i) {
-        refill();
-        uint32_t pat;
-        if ((buf & 1ull) == 0ull)      { pat = 0u; buf >>= 1; have -= 1; }
-        else if ((buf & 2ull) == 0ull) { pat = (buf & 4ull) ? (tp | PfxTraits<DT>::kSign) : tp; buf >>= 3; have -= 3; }
-        else {
-            buf >>= 2; have -= 2;
-            refill();                                            // now at least 32 bits: the whole value
-            pat = (uint32_t)buf & (DT == LGN_F32 ? 0xFFFFFFFFu : 0xFFFFu);
-            buf >>= PfxTraits<DT>::kWidth; have -= PfxTraits<DT>::kWidth;
+    for (uint32_t j = 0; j < LGN_PREFIX_BLOCK; j += 32) {
+        const uint64_t ic = i0 + j;
+        const uint32_t cnt = ic >= i1 ? 0u : (i1 - ic < 32u ? (uint32_t)(i1 - ic) : 32u);
+        for (uint32_t k = 0; k < cnt; ++k) {
+            refill();
+            uint32_t pat;
+            if ((buf & 1ull) == 0ull)      { pat = 0u; buf >>= 1; have -= 1; }
+            else if ((buf & 2ull) == 0ull) { pat = (buf & 4ull) ? (tp | PfxTraits<DT>::kSign) : tp; buf >>= 3; have -= 3; }
+            else {
+                buf >>= 2; have -= 2;
+                refill();                                        // now at least 32 bits: the whole value
+                pat = (uint32_t)buf & (DT == LGN_F32 ? 0xFFFFFFFFu : 0xFFFFu);
+                buf >>= PfxTraits<DT>::kWidth; have -= PfxTraits<DT>::kWidth;
+            }
+            tile[warp][lane][k] = pat;
         }
-        if (DT == LGN_F32) static_cast<uint32_t *>(out)[i] = pat;
-        else               static_cast<uint16_t *>(out)[i] = (uint16_t)pat;
+        __syncwarp();
+        #pragma unroll 4
+        for (int r = 0; r < 32; ++r) {                           // row r = block b0 + r, elements j .. j+31
+            const uint64_t i = (b0 + r) * LGN_PREFIX_BLOCK + j + lane;
+            if (b0 + r < nblocks && i < n) {
+                const uint32_t v = tile[warp][r][lane];
+                if (DT == LGN_F32) static_cast<uint32_t *>(out)[i] = v;
+                else               static_cast<uint16_t *>(out)[i] = (uint16_t)v;
+            }
+        }
+        __syncwarp();
     }
 }
 
@@ -376,9 +401,9 @@ extern "C" lgn_status lgn_prefix_decode(const uint32_t *stream_dev, const uint64
     if (n == 0) return LGN_OK;
     const uint64_t nb = lgn_prefix_blocks(n);
     const float tau_used = dt == LGN_BF16 ? snap_threshold_bf16(tau) : snap_threshold_f32(tau);
-    const unsigned grid = (unsigned)((nb + 127) / 128);
+    const unsigned grid = (unsigned)((nb + kDecThreads - 1) / kDecThreads);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (dt == LGN_F32) prefix_decode_kernel<LGN_F32><<<grid, 128, 0, st>>>(stream_dev, off_dev, n, nb, tau_used, tau_from_dev, out_dev);
-    else               prefix_decode_kernel<LGN_BF16><<<grid, 128, 0, st>>>(stream_dev, off_dev, n, nb, tau_used, tau_from_dev, out_dev);
+    if (dt == LGN_F32) prefix_decode_kernel<LGN_F32><<<grid, kDecThreads, 0, st>>>(stream_dev, off_dev, n, nb, tau_used, tau_from_dev, out_dev);
+    else               prefix_decode_kernel<LGN_BF16><<<grid, kDecThreads, 0, st>>>(stream_dev, off_dev, n, nb, tau_used, tau_from_dev, out_dev);
     return cudaGetLastError() == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
 }

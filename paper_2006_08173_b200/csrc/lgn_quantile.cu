@@ -96,16 +96,41 @@ __device__ __forceinline__ unsigned long long cta_exclusive_scan(unsigned long l
     return incl - v + (warp ? sm[warp - 1] : 0ull);
 }
 
-// Finds the bin that holds rank `rank` (1-based) among `nbins` counts; thread t owns nbins/kQThreads consecutive bins.
-// Returns true in exactly one thread, with *bin and *rank_in_bin set.
+// Sum of the PER consecutive counts a thread owns, with 16-byte loads (all in flight together).
 template <int PER>
-__device__ __forceinline__ bool locate(const uint32_t *hist, unsigned long long rank, unsigned long long before,
-                                       uint32_t *bin, unsigned long long *rank_in_bin) {
-    unsigned long long cum = before;
-    for (int k = 0; k < PER; ++k) {
-        const uint32_t c = hist[threadIdx.x * PER + k];
-        if (rank > cum && rank <= cum + c) { *bin = threadIdx.x * PER + k; *rank_in_bin = rank - cum; return true; }
-        cum += c;
+__device__ __forceinline__ unsigned long long own_sum(const uint32_t *hist) {
+    const uint4 *p = reinterpret_cast<const uint4 *>(hist + (size_t)threadIdx.x * PER);
+    unsigned long long s = 0;
+    #pragma unroll
+    for (int k = 0; k < PER / 4; ++k) { const uint4 v = p[k]; s += (unsigned long long)v.x + v.y + v.z + v.w; }
+    return s;
+}
+
+// Finds the bin that holds rank `rank` (1-based, 1 <= rank <= total): the thread whose PER
+// bins contain it announces itself, then warp 0 scans those bins 32 at a time.  Returns
+// true in one lane of warp 0, with *bin and *rank_in_bin set.  All threads must call.
+template <int PER>
+__device__ __forceinline__ bool locate(const uint32_t *hist, unsigned long long rank, unsigned long long mine,
+                                       unsigned long long before, uint32_t *bin, unsigned long long *rank_in_bin) {
+    __shared__ uint32_t sm_owner;
+    __shared__ unsigned long long sm_before;
+    if (rank > before && rank <= before + mine) { sm_owner = threadIdx.x; sm_before = before; }
+    __syncthreads();
+    if (threadIdx.x >= 32) return false;
+    const int lane = threadIdx.x;
+    const uint32_t base = sm_owner * PER;
+    unsigned long long cum = sm_before;
+    for (int j = 0; j < PER; j += 32) {
+        const uint32_t c = hist[base + j + lane];
+        unsigned long long incl = c;
+        #pragma unroll
+        for (int d = 1; d < 32; d <<= 1) { const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, incl, d); if (lane >= d) incl += t; }
+        const bool hit = rank > cum + incl - c && rank <= cum + incl;
+        if (__any_sync(0xFFFFFFFFu, hit)) {
+            if (hit) { *bin = base + j + lane; *rank_in_bin = rank - (cum + incl - c); }
+            return hit;
+        }
+        cum += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
     return false;
 }
@@ -115,8 +140,8 @@ __global__ void __launch_bounds__(kQThreads)
 quantile_pick_top_kernel(const uint32_t *hist_top, double q, QCtl *ctl, lgn_quantile_t *out) {
     __shared__ unsigned long long sm[32];
     constexpr int PER = kQTopBins / kQThreads;
-    unsigned long long mine = 0, nnz;
-    for (int k = 0; k < PER; ++k) mine += hist_top[threadIdx.x * PER + k];
+    unsigned long long nnz;
+    const unsigned long long mine = own_sum<PER>(hist_top);
     const unsigned long long before = cta_exclusive_scan(mine, sm, &nnz);
     if (nnz == 0) {
         if (threadIdx.x == 0) { ctl->nnz = 0; ctl->rank_in_bin = 0; ctl->bin = 0; out->value = 0.f; out->pad = 0; out->nnz = 0; }
@@ -127,7 +152,7 @@ quantile_pick_top_kernel(const uint32_t *hist_top, double q, QCtl *ctl, lgn_quan
     if (r > nnz) r = nnz;
     uint32_t bin;
     unsigned long long rib;
-    if (locate<PER>(hist_top, r, before, &bin, &rib)) {
+    if (locate<PER>(hist_top, r, mine, before, &bin, &rib)) {
         ctl->nnz = nnz; ctl->bin = bin; ctl->rank_in_bin = rib;
         if (DT == LGN_BF16) { out->value = u2f(bin << 16); out->pad = 0; out->nnz = nnz; }
     }
@@ -145,12 +170,12 @@ quantile_pick_low_kernel(const uint32_t *hist_low, const QCtl *ctl, lgn_quantile
     __shared__ unsigned long long sm[32];
     if (ctl->nnz == 0) return;
     constexpr int PER = kQLowBins / kQThreads;
-    unsigned long long mine = 0, total;
-    for (int k = 0; k < PER; ++k) mine += hist_low[threadIdx.x * PER + k];
+    unsigned long long total;
+    const unsigned long long mine = own_sum<PER>(hist_low);
     const unsigned long long before = cta_exclusive_scan(mine, sm, &total);
     uint32_t low;
     unsigned long long rib;
-    if (locate<PER>(hist_low, ctl->rank_in_bin, before, &low, &rib)) {
+    if (locate<PER>(hist_low, ctl->rank_in_bin, mine, before, &low, &rib)) {
         out->value = u2f((ctl->bin << 16) | low); out->pad = 0; out->nnz = ctl->nnz;
     }
 }

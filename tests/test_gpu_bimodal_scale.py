@@ -17,7 +17,7 @@ SIZES = [1, 3, 1023, 40_000, 2 ** 20 + 7]
 def close(got, want):
     assert got["nnz"] == want["nnz"]
     scale = max(abs(want["mu"]), want["sigma"], 1e-300)
-    small = want["nnz"] <= 3                                   # one to three samples: see DESIGN tolerances
+    small = want["nnz"] <= 3                                   # one to three samples: 1e-5 of max(|mu|, 1), 1e-4 absolute on sigma
     assert abs(got["mu"] - want["mu"]) <= REL_TOL * (max(abs(want["mu"]), 1.0) if small else scale)
     assert abs(got["sigma"] - want["sigma"]) <= (1e-4 if small else REL_TOL * max(want["sigma"], 1e-300)) \
         or (want["sigma"] == 0.0 and got["sigma"] <= 1e-6)

@@ -173,3 +173,42 @@ def test_grouped_path_is_deterministic(lgn):
         o2, r2 = run_group(lgn, tensors, lspecs)
         assert r1 == r2
         assert all(torch.equal(a, b) for a, b in zip(o1, o2))
+
+
+def test_host_buffer_form_in_several_groups(lgn):
+    """Enough input (5 x 40 MB) for the host form to run its layers in three pipelined
+    groups, of mixed kinds: every output and result must be what one grouped call on
+    device tensors gives."""
+    n = 10_000_000
+    gs = [synth.lognormal_tensor(n + 1000 * k, -12.0 + k, 2.0, 0.4, seed=40 + k) for k in range(5)]
+    kinds = [dict(mode=lgn.MODE_PRUNE, S=0.8), dict(mode=lgn.MODE_QUANTIZE, nbits=6, rounding=lgn.ROUND_STOCHASTIC),
+             dict(mode=lgn.MODE_PRUNE, S=0.6), dict(mode=lgn.MODE_PRUNE, S=0.9),
+             dict(mode=lgn.MODE_QUANTIZE, nbits=5, rounding=lgn.ROUND_NEAREST)]
+
+    def out_like(g, kd, device):
+        if kd["mode"] == lgn.MODE_PRUNE:
+            return torch.empty(g.shape, dtype=g.dtype, device=device)
+        return torch.zeros(lgn.lgn_codes_bytes(g.numel(), kd["nbits"]), dtype=torch.uint8, device=device)
+
+    hin = [g.pin_memory() for g in gs]
+    hout = [out_like(g, kd, "cpu").pin_memory() for g, kd in zip(gs, kinds)]
+    hl = [lgn.make_host_layer(a, b, kd["mode"], seed=7 + k, **{x: y for x, y in kd.items() if x != "mode"})
+          for k, (a, b, kd) in enumerate(zip(hin, hout, kinds))]
+    buf = torch.empty(lgn.lgn_host_staging_bytes(hl) + 256, dtype=torch.uint8, device="cuda")
+    buf = buf[(-buf.data_ptr()) % 256:]
+    res_h = lgn.lgn_compress_layers_host(hl, buf)
+
+    dg = [g.cuda() for g in gs]
+    dout = [out_like(g, kd, "cuda") for g, kd in zip(dg, kinds)]
+    dl = [lgn.make_layer(a, b, kd["mode"], seed=7 + k, **{x: y for x, y in kd.items() if x != "mode"})
+          for k, (a, b, kd) in enumerate(zip(dg, dout, kinds))]
+    res = lgn.new_results(5, "cuda")
+    lgn.lgn_compress_layers(dl, res, lgn.new_workspace([g.numel() for g in dg], "cuda"))
+    torch.cuda.synchronize()
+    res_d = lgn.read_results(res, 5)
+    for k in range(5):
+        assert res_h[k]["status"] == 0
+        for key in ("n", "nnz", "tau", "fmt"):
+            assert res_h[k][key] == res_d[k][key], (k, key)
+        assert abs(res_h[k]["mu"] - res_d[k]["mu"]) <= 1e-9 * abs(res_d[k]["mu"])
+        assert torch.equal(hout[k].view(torch.uint8), dout[k].cpu().view(torch.uint8)), k
