@@ -67,9 +67,28 @@ LGN_HD double solve_threshold_u(double s, double Sp) {
     double q = Sp / (1.0 - Sp);
     double u = (q > 0.0 && q < 1e300) ? s * log(q) * 0.5875 + 1.0 : 0.0;
     if (!(u > lo && u < hi)) u = 0.0;
+    const bool well_conditioned = Sp >= 1e-4 && Sp <= 1.0 - 1e-4;
+    // A few Newton steps in fp32 first (an fp32 erfc costs a tenth of an fp64 one): they bring
+    // the start to within about 1e-5 of the root, so the fp64 iteration below needs two or
+    // three evaluations instead of five or six.  Only a better starting point: every decision
+    // about the result is taken in fp64.
+    if (Sp >= 1e-3 && Sp <= 1.0 - 1e-3 && s >= 0.05 && s <= 8.0) {
+        float uf = (float)u;
+        const float sf = (float)s, target = (float)Sp;
+        for (int it = 0; it < 4; ++it) {
+            const float ex = 0.5f * sf * sf - uf;
+            if (!(ex < 60.0f)) break;
+            const float a = 0.5f * erfcf(-uf / sf * 0.70710678f);
+            const float b = expf(ex) * 0.5f * erfcf(-(uf - sf * sf) / sf * 0.70710678f);
+            if (!(b > 1e-20f)) break;
+            const float un = uf - (a - b - target) / b;
+            if (!(un > (float)lo && un < (float)hi)) break;
+            uf = un;
+        }
+        if (uf > (float)lo && uf < (float)hi) u = (double)uf;
+    }
     double prev_step = 1e300;
     bool prev_newton = false;
-    const bool well_conditioned = Sp >= 1e-4 && Sp <= 1.0 - 1e-4;
     for (int it = 0; it < 200; ++it) {
         double F, dF;
         pruned_fraction(u, s, F, dF);

@@ -115,29 +115,37 @@ static_assert(sizeof(PfxCtl) == 256, "control block");
 constexpr unsigned long long kPfxAggregate = 1ull, kPfxInclusive = 2ull;
 constexpr uint32_t kPfxMaxPolls = 1u << 20;
 
-__device__ __forceinline__ unsigned long long ld_acquire64(const unsigned long long *p) {
+// A block's state word carries everything a successor needs (flag and length in one
+// aligned 64-bit word) and nothing else is read through it, so relaxed accesses at
+// gpu scope are enough.
+__device__ __forceinline__ unsigned long long ld_state(const unsigned long long *p) {
     unsigned long long v;
-    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void st_release64(unsigned long long *p, unsigned long long v) {
-    asm volatile("st.release.gpu.global.u64 [%0], %1;" :: "l"(p), "l"(v) : "memory");
+__device__ __forceinline__ void st_state(unsigned long long *p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" :: "l"(p), "l"(v) : "memory");
 }
 
-// OR the low `len` bits of x (its other bits are zero) into the image at bit position `at`.
-__device__ __forceinline__ void pfx_or64(uint32_t *img, uint32_t at, unsigned long long x) {
-    const uint32_t s = at & 31u, w = at >> 5;
-    const uint32_t lo = (uint32_t)x, hi = (uint32_t)(x >> 32);
-    const uint32_t w0 = lo << s, w1 = __funnelshift_l(lo, hi, s), w2 = __funnelshift_l(hi, 0u, s);
-    if (w0) atomicOr(img + w, w0);
-    if (w1) atomicOr(img + w + 1, w1);
-    if (w2) atomicOr(img + w + 2, w2);
+// OR a word into the image unless it is zero: a compare and a predicated shared-memory
+// reduction, no branch (most words of most lanes are zero).
+__device__ __forceinline__ void pfx_or_word(uint32_t addr, uint32_t v) {
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %1, 0;\n\t@p red.shared.or.b32 [%0], %1;\n\t}"
+                 :: "r"(addr), "r"(v) : "memory");
 }
-__device__ __forceinline__ void pfx_or32(uint32_t *img, uint32_t at, uint32_t x) {
-    const uint32_t s = at & 31u, w = at >> 5;
-    const uint32_t w0 = x << s, w1 = __funnelshift_l(x, 0u, s);
-    if (w0) atomicOr(img + w, w0);
-    if (w1) atomicOr(img + w + 1, w1);
+
+// OR the bits of x (bits above its length are zero) into the image at bit position `at`.
+__device__ __forceinline__ void pfx_or64(uint32_t img_addr, uint32_t at, unsigned long long x) {
+    const uint32_t s = at & 31u, a = img_addr + (at >> 5) * 4u;
+    const uint32_t lo = (uint32_t)x, hi = (uint32_t)(x >> 32);
+    pfx_or_word(a, lo << s);
+    pfx_or_word(a + 4u, __funnelshift_l(lo, hi, s));
+    pfx_or_word(a + 8u, __funnelshift_l(hi, 0u, s));
+}
+__device__ __forceinline__ void pfx_or32(uint32_t img_addr, uint32_t at, uint32_t x) {
+    const uint32_t s = at & 31u, a = img_addr + (at >> 5) * 4u;
+    pfx_or_word(a, x << s);
+    pfx_or_word(a + 4u, __funnelshift_l(x, 0u, s));
 }
 
 template <int DT, bool PRUNE>
@@ -148,6 +156,7 @@ prefix_encode_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host
     constexpr uint32_t kSign = PfxTraits<DT>::kSign;
     constexpr uint32_t W = PfxTraits<DT>::kWidth;
     __shared__ uint32_t img[kPfxImageWords];
+    __shared__ uint32_t pay[kPfxPerThread][kPfxThreads];         // the threads' (pruned) patterns, one column each
     __shared__ uint32_t sm_scan[kPfxWarps];
     __shared__ unsigned long long sm_ticket, sm_excl;
     const float tau = pfx_tau(tau_host, tau_from);
@@ -180,6 +189,7 @@ prefix_encode_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host
             q += (in ? 1u : 0u) + (nz ? 1u : 0u) + (al ? 1u : 0u);
             if (nz && !al) vm |= 1u << k;
             cuts |= (unsigned long long)q << (5 * k);
+            pay[k][threadIdx.x] = pat;
         }
         const uint32_t bits = q + W * __popc(vm);
 
@@ -197,26 +207,29 @@ prefix_encode_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host
         for (int w = 0; w < kPfxWarps; ++w) { const uint32_t t = sm_scan[w]; if (w < warp) pos += t; total += t; }
         const uint32_t words = (total + 31u) >> 5;
         if (threadIdx.x == 0) {
-            if (b == 0) { st_release64(state, ((unsigned long long)words << 2) | kPfxInclusive); sm_excl = 0ull; }
-            else        st_release64(state + b, ((unsigned long long)words << 2) | kPfxAggregate);
+            if (b == 0) { st_state(state, ((unsigned long long)words << 2) | kPfxInclusive); sm_excl = 0ull; }
+            else        st_state(state + b, ((unsigned long long)words << 2) | kPfxAggregate);
         }
         for (uint32_t k = threadIdx.x; k < words + 2u; k += kPfxThreads) img[k] = 0u;
         __syncthreads();
 
         // the thread's bits into the image
+        const uint32_t img_addr = (uint32_t)__cvta_generic_to_shared(img);
+        // One trip per value of the thread (a warp makes as many trips as its busiest lane
+        // has values, about three at 8 % values, instead of eight trips over the elements);
+        // the value is fetched from the thread's own column of `pay` by its index.
         uint32_t cur = pos, done = 0u;
-        #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            if (vm & (1u << k)) {
-                const uint32_t cut = (uint32_t)(cuts >> (5 * k)) & 31u;
-                const uint32_t plen = cut - done;                // 2..26: ends with the value's "11"
-                const uint32_t piece = (sb >> done) & ((1u << plen) - 1u);
-                pfx_or64(img, cur, (unsigned long long)piece | ((unsigned long long)p[k] << plen));
-                cur += plen + W;
-                done = cut;
-            }
+        for (uint32_t m = vm; m; m &= m - 1u) {
+            const int k = __ffs(m) - 1;
+            const uint32_t cut = (uint32_t)(cuts >> (5 * k)) & 31u;
+            const uint32_t plen = cut - done;                    // 2..26: ends with the value's "11"
+            const uint32_t piece = (sb >> done) & ((1u << plen) - 1u);
+            const uint32_t val = pay[k][threadIdx.x];
+            pfx_or64(img_addr, cur, (unsigned long long)piece | ((unsigned long long)val << plen));
+            cur += plen + W;
+            done = cut;
         }
-        if (q > done) pfx_or32(img, cur, sb >> done);
+        if (q > done) pfx_or32(img_addr, cur, sb >> done);
 
         // warp 0: first word of this block = sum of the lengths of all earlier blocks
         if (warp == 0 && b > 0) {
@@ -227,7 +240,7 @@ prefix_encode_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host
                 unsigned long long v = kPfxInclusive;            // before block 0: an inclusive prefix of 0
                 uint32_t polls = 0;
                 for (;;) {
-                    if (idx >= 0) v = ld_acquire64(state + idx);
+                    if (idx >= 0) v = ld_state(state + idx);
                     if (!__any_sync(0xFFFFFFFFu, (v & 3ull) == 0ull)) break;
                     const bool stop = ++polls > kPfxMaxPolls || *(volatile uint32_t *)&ctl->error != 0u;
                     if (__any_sync(0xFFFFFFFFu, stop)) { fail = true; break; }
@@ -244,7 +257,7 @@ prefix_encode_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host
             }
             if (lane == 0) {
                 if (fail) { atomicExch(&ctl->error, 1u); sm_excl = ~0ull; }
-                else      { st_release64(state + b, ((excl + words) << 2) | kPfxInclusive); sm_excl = excl; }
+                else      { st_state(state + b, ((excl + words) << 2) | kPfxInclusive); sm_excl = excl; }
             }
         }
         __syncthreads();                                         // the image is complete, the offset known
