@@ -68,6 +68,9 @@ for _lg in (26, 28):
                                                          dtype="f32" if _dt == "fp32" else "bf16", mode="prune")
         WORKLOADS[f"max_scale_fp6_{_dt}_2p{_lg}"] = dict(net="aux", kind="maxscale", log2n=_lg, nbits=6,
                                                          dtype="f32" if _dt == "fp32" else "bf16", mode="quant")
+        for _k in ("stats", "apply_prune", "apply_fp6"):           # the entry points of the steady-state iterations
+            WORKLOADS[f"{_k}_{_dt}_2p{_lg}"] = dict(net="aux", kind=_k, log2n=_lg, nbits=6,
+                                                    dtype="f32" if _dt == "fp32" else "bf16", mode=_k)
         WORKLOADS[f"quantile_{_dt}_2p{_lg}"] = dict(net="aux", kind="quantile", log2n=_lg,
                                                     dtype="f32" if _dt == "fp32" else "bf16", mode="quantile")
         WORKLOADS[f"prefix_decode_{_dt}_2p{_lg}"] = dict(net="aux", kind="prefix", decode=True, log2n=_lg,
@@ -364,6 +367,29 @@ def run_aux(args):
         alg_bytes = n * (w["nbits"] / 8.0 + esize)
         call = lambda: lgn.lgn_dequantize(codes, n, fmt, out)
         kernel = "dequantize_kernel"
+    elif w["kind"] in ("stats", "apply_prune", "apply_fp6"):
+        # one entry point alone: the statistics pass, or an apply pass with a cached threshold / format
+        g = synth.lognormal_tensor(n, -12.0, 2.0, 0.5, 0, dtype, str(dev))
+        st = lgn.lgn_stats(g)
+        if w["kind"] == "stats":
+            ws = lgn.new_workspace([n], dev)
+            out = torch.empty(64, dtype=torch.uint8, device=dev)
+            call = lambda: lgn.lgn_stats_async(g, out, ws)
+            alg_bytes = float(n * esize)
+            kernel = "compress_kernel (statistics only)"
+            launches = lgn.lgn_launches_per_call(1)
+        elif w["kind"] == "apply_prune":
+            tau = lgn.lgn_threshold(st["mu"], st["sigma"], 1.0 - st["nnz"] / st["n"], 0.85)
+            out = torch.empty_like(g)
+            call = lambda: lgn.lgn_prune(g, tau, 1, out)
+            alg_bytes = 2.0 * n * esize
+            kernel = "prune_kernel"
+        else:
+            fmt = lgn.lgn_fp_format(st["mu"], st["sigma"], w["nbits"])
+            out = torch.empty(lgn.lgn_codes_bytes(n, w["nbits"]), dtype=torch.uint8, device=dev)
+            call = lambda: lgn.lgn_quantize(g, fmt, lgn.ROUND_STOCHASTIC, 1, out)
+            alg_bytes = n * (esize + w["nbits"] / 8.0)
+            kernel = "quantize_kernel"
     elif w["kind"] == "quantile":
         g = synth.lognormal_tensor(n, -12.0, 2.0, 0.5, 0, dtype, str(dev))
         ws = torch.empty(lgn.lgn_quantile_workspace_bytes(), dtype=torch.uint8, device=dev)
