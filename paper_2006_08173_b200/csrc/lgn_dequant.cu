@@ -88,12 +88,15 @@ dequantize_kernel(const uint32_t *__restrict__ codes, void *__restrict__ out, ui
             for (int k = 0; k < NW; ++k) v[k] = __funnelshift_r(r[k], r[k + 1], sh);
             v[NW] = 0u;
             Chunk o;
-            #pragma unroll
-            for (int e = 0; e < C; ++e) {
-                const uint32_t b = decode_at<NBITS>(v, e * NBITS, p);
-                if (ODT == LGN_F32) o.w[e] = b;
-                else if ((e & 1) == 0) o.w[e >> 1] = b >> 16;
-                else o.w[e >> 1] |= b & 0xFFFF0000u;
+            if constexpr (ODT == LGN_F32) {
+                #pragma unroll
+                for (int e = 0; e < C; ++e) o.w[e] = decode_at<NBITS>(v, e * NBITS, p);
+            } else {
+                #pragma unroll
+                for (int e = 0; e < C; e += 2) {                 // the upper halves of two fp32 patterns: one byte permute
+                    const uint32_t b0 = decode_at<NBITS>(v, e * NBITS, p), b1 = decode_at<NBITS>(v, (e + 1) * NBITS, p);
+                    o.w[e >> 1] = __byte_perm(b0, b1, 0x7632);
+                }
             }
             if (full) store_chunk<ODT, true>(out, i, n, o);
             else      store_chunk<ODT, false>(out, i, n, o);
