@@ -535,7 +535,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample-elems", type=int, default=230_000_000)
+    ap.add_argument("--cpu-sample-elems", type=int, default=300_000_000)
     ap.add_argument("--ref-sample-elems", type=int, default=33_000_000)
     args = ap.parse_args()
     if args.warmup < 3:
