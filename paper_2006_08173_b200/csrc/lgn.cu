@@ -122,6 +122,10 @@ constexpr int kBlobBytes = 3840;
 struct Blob { uint4 v[kBlobBytes / 16]; };
 
 __global__ void upload_kernel(const __grid_constant__ Blob blob, uint4 *dst, int nvec) {
+    // A compute kernel launched behind this one with programmatic stream
+    // serialisation may be scheduled now; it waits (griddepcontrol.wait) for this
+    // grid to finish and its stores to be visible before it reads the image.
+    asm volatile("griddepcontrol.launch_dependents;");
     for (int i = threadIdx.x; i < nvec; i += blockDim.x) dst[i] = blob.v[i];
 }
 
@@ -368,6 +372,10 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
     __shared__ uint32_t sm_flag;
     constexpr bool kSpecial = DT != kAny;
 
+    // Launched with programmatic stream serialisation behind the last set-up
+    // launch: the CTAs may already be resident while that launch runs, and wait
+    // here until it has finished and the workspace image is visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (blockIdx.x == 0) {                       // layers with no elements have no tiles: answer here
         for (int k = threadIdx.x; k < num_layers; k += kThreads) {
             const LayerState &L = states[k];
@@ -743,7 +751,17 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
     uint32_t a_items = total_items;
     Partial *a_partials = reinterpret_cast<Partial *>(base + w.partials);
     void *args[] = { &a_hdr, &a_states, &a_dyn, &a_segs, &a_L, &a_items, &a_partials };
-    if (cudaLaunchKernel(fn, dim3((unsigned)grid), dim3(kThreads), args, 0, stream) != cudaSuccess) return LGN_ERR_CUDA;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;     // overlap the launch with the set-up launch before it
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelExC(&cfg, fn, args) != cudaSuccess) return LGN_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? LGN_OK : LGN_ERR_CUDA;
 }
 
