@@ -118,15 +118,34 @@ static bool ws_layout(const uint64_t *n_per_layer, int L, WsLayout &w) {
 // ------------------------------------------------------------------ set-up launch
 // Host bytes travel to the device inside the kernel parameter block: no pinned
 // staging buffer, no synchronous copy, ordered on the stream like any launch.
+// Two sizes: an image of up to kBlobBytes goes in one small launch; a larger one
+// (more than a dozen layers) in launches of kBigBlobBytes each, so that a call with
+// a hundred layers still has a single set-up launch.
 constexpr int kBlobBytes = 3840;
-struct Blob { uint4 v[kBlobBytes / 16]; };
+constexpr int kBigBlobBytes = 30720;
+template <int BYTES> struct BlobT { uint4 v[BYTES / 16]; };
 
-__global__ void upload_kernel(const __grid_constant__ Blob blob, uint4 *dst, int nvec) {
+template <int BYTES>
+__global__ void upload_kernel(const __grid_constant__ BlobT<BYTES> blob, uint4 *dst, int nvec) {
     // A compute kernel launched behind this one with programmatic stream
     // serialisation may be scheduled now; it waits (griddepcontrol.wait) for this
     // grid to finish and its stores to be visible before it reads the image.
     asm volatile("griddepcontrol.launch_dependents;");
     for (int i = threadIdx.x; i < nvec; i += blockDim.x) dst[i] = blob.v[i];
+}
+
+template <int BYTES>
+static void upload_image(const unsigned char *image, size_t used, unsigned char *base, cudaStream_t stream) {
+    for (size_t off = 0; off < used; off += BYTES) {
+        BlobT<BYTES> blob;
+        const size_t nb = used - off < (size_t)BYTES ? used - off : (size_t)BYTES;
+        memcpy(blob.v, image + off, nb);                    // nb is a multiple of 16
+        upload_kernel<BYTES><<<1, BYTES >= 8192 ? 256 : 128, 0, stream>>>(blob, reinterpret_cast<uint4 *>(base + off), (int)(nb / 16));
+    }
+}
+
+static int upload_launches(size_t used) {
+    return used <= (size_t)kBlobBytes ? 1 : (int)((used + kBigBlobBytes - 1) / kBigBlobBytes);
 }
 
 // The uploaded image is [header | states | dyn | segments]: it ends after the
@@ -734,12 +753,8 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
     memcpy(image.data() + w.segs, segs.data(), sizeof(Segment) * segs.size());
     const size_t used = upload_bytes(w, L);
     unsigned char *base = static_cast<unsigned char *>(ws);
-    for (size_t off = 0; off < used; off += kBlobBytes) {
-        Blob blob;
-        const size_t nb = used - off < (size_t)kBlobBytes ? used - off : (size_t)kBlobBytes;
-        memcpy(blob.v, image.data() + off, nb);             // nb is a multiple of 16
-        upload_kernel<<<1, 128, 0, stream>>>(blob, reinterpret_cast<uint4 *>(base + off), (int)(nb / 16));
-    }
+    if (used <= (size_t)kBlobBytes) upload_image<kBlobBytes>(image.data(), used, base, stream);
+    else                            upload_image<kBigBlobBytes>(image.data(), used, base, stream);
     if (cudaGetLastError() != cudaSuccess) return LGN_ERR_CUDA;
 
     if ((uint32_t)grid > total_items) grid = (int)(total_items ? total_items : 1u);
@@ -794,7 +809,7 @@ extern "C" int lgn_launches_per_call(int num_layers) {
     std::vector<uint64_t> ns((size_t)num_layers, 1);
     WsLayout w;
     if (!ws_layout(ns.data(), num_layers, w)) return 0;
-    return (int)((upload_bytes(w, num_layers) + kBlobBytes - 1) / kBlobBytes) + 1;
+    return upload_launches(upload_bytes(w, num_layers)) + 1;
 }
 
 extern "C" size_t lgn_codes_bytes(uint64_t n, int nbits) {
