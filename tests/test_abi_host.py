@@ -51,6 +51,11 @@ def test_sizes(lgn, oracle):
     assert w1 % 256 == 0
     assert lgn.lgn_workspace_bytes([]) > 0
     assert lgn.lgn_workspace_bytes([2 ** 50]) == 0           # too large: reported as 0
+    # launches per grouped call: one set-up launch up to about 110 layers, then one more per 112 or so
+    assert lgn.lgn_launches_per_call(0) == 0
+    assert [lgn.lgn_launches_per_call(L) for L in (1, 20, 53, 100)] == [2, 2, 2, 2]
+    counts = [lgn.lgn_launches_per_call(L) for L in range(1, 400)]
+    assert counts == sorted(counts) and counts[-1] == 5
 
 
 @pytest.mark.parametrize("sigma", [1e-3, 0.3, 1.0, 1.5, 2.0, 3.0, 4.0, 5.5, 8.0, 25.0, 40.0])

@@ -120,6 +120,24 @@ def test_mixed_modes_dtypes_and_empty_layers(lgn, oracle):
     check_group(lgn, oracle, tensors, specs)
 
 
+def test_many_layers_in_one_call(lgn, oracle):
+    """150 small layers in one call: the descriptors of that many layers no longer
+    fit one set-up launch (its parameter block holds about 110 layers), so this
+    call takes two; every layer is still checked in full against the oracle."""
+    L = 150
+    assert lgn.lgn_launches_per_call(L) == 3 and lgn.lgn_launches_per_call(100) == 2
+    tensors, specs = [], []
+    for k in range(L):
+        dt = torch.bfloat16 if k % 3 == 2 else torch.float32
+        tensors.append(synth.lognormal_tensor(500 + 37 * k, -14.0 + 0.03 * k, 1.5 + 0.01 * k, 0.3, 100 + k,
+                                              dtype=dt, device="cuda"))
+        if k % 2:
+            specs.append(dict(mode="quant", nbits=5 + (k % 4 == 3), rounding=(k // 2) % 2, seed=k))
+        else:
+            specs.append(dict(mode="prune", S=(0.5, 0.7, 0.85, 0.9)[(k // 2) % 4], seed=k))
+    check_group(lgn, oracle, tensors, specs)
+
+
 # ------------------------------------------------------------------ edge-case stress
 EDGE_INPUTS = [
     dict(n=1), dict(n=3), dict(n=1023), dict(n=2 ** 20 + 7),
