@@ -138,6 +138,26 @@ def test_many_layers_in_one_call(lgn, oracle):
     check_group(lgn, oracle, tensors, specs)
 
 
+def test_call_is_ordered_after_earlier_work_on_its_stream(lgn):
+    """The compute kernel may become resident while the set-up launch before it still
+    runs; it must all the same see what earlier kernels on the stream wrote.  The
+    input is overwritten by copies enqueued right before the call, with no
+    synchronisation in between, and the output must be that of the new contents."""
+    n = 2 ** 25 + 5
+    a = synth.lognormal_tensor(n, -12.0, 2.0, 0.4, 31, device="cuda")
+    b = synth.lognormal_tensor(n, -10.0, 2.5, 0.2, 32, device="cuda")
+    specs = [dict(mode="prune", S=0.8, seed=9)]
+    (want,), (want_res,) = run_group(lgn, [b.clone()], specs)
+    g = a.clone()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        g.copy_(a)
+        g.copy_(b)                                   # still running when the call below is enqueued
+        (got,), (res,) = run_group(lgn, [g], specs)
+        assert res["status"] == 0 and res["tau"] == want_res["tau"]
+        assert torch.equal(got.view(torch.int32), want.view(torch.int32))
+
+
 # ------------------------------------------------------------------ edge-case stress
 EDGE_INPUTS = [
     dict(n=1), dict(n=3), dict(n=1023), dict(n=2 ** 20 + 7),
