@@ -105,21 +105,82 @@ def read_peak():
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons of one GPU, sampled while the timed region runs."""
+    """SM clock and throttle reasons of one GPU, sampled while work runs: NVML polled from a
+    thread every few milliseconds (a timed region of 20 ms still gets samples), or
+    `nvidia-smi -lms` when NVML's Python module is missing.  Reads settings only."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
-    def __init__(self, index: int):
-        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+    def __init__(self, index: int, period_s: float = 0.004):
+        self.samples = []                # (time, sm_mhz, set of reasons)
+        self.max_mhz = None
+        self.marks = {}
+        self.p = self.f = self.thread = None
+        self.how = "nvml"
         try:
-            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                       "-lms", "100", "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            # NVML orders devices by PCI bus id; CUDA_VISIBLE_DEVICES may renumber them
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if vis:
+                ent = [v.strip() for v in vis.split(",") if v.strip()]
+                if index < len(ent) and ent[index].isdigit():
+                    phys = int(ent[index])
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.stop_flag = False
+            import threading
+            self.period = period_s
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
         except Exception:
-            self.p = None
+            self.how = "nvidia-smi"
+            self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            try:
+                self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                           "-lms", "20", "-i", str(index)], stdout=self.f, stderr=subprocess.DEVNULL)
+            except Exception:
+                self.p = None
+
+    def _poll(self):
+        nv = self.nv
+        bits = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown,
+                "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+                "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap}
+        while not self.stop_flag:
+            try:
+                mhz = float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                self.samples.append((time.perf_counter(), mhz, {k for k, b in bits.items() if mask & b}))
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def mark(self, name: str):
+        self.marks[name] = time.perf_counter()
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "how": self.how}
+        if self.thread is not None:
+            self.stop_flag = True
+            self.thread.join(timeout=2)
+            t0, t1 = self.marks.get("timed_begin"), self.marks.get("timed_end")
+            load = [x for x in self.samples if self.marks.get("load_begin", 0) <= x[0] <= self.marks.get("load_end", 1e300)]
+            timed = [x for x in load if t0 is not None and t1 is not None and t0 <= x[0] <= t1]
+            if load:
+                reasons = set()
+                for x in load:
+                    reasons |= x[2]
+                out.update(sm_mhz=statistics.median(x[1] for x in load), sm_max_mhz=self.max_mhz, samples=len(load),
+                           samples_in_timed_region=len(timed), reasons=sorted(reasons))
+                if timed:
+                    out["sm_mhz_timed_region"] = statistics.median(x[1] for x in timed)
+            return out
         if self.p is None:
             return out
         self.p.terminate()
@@ -130,7 +191,6 @@ class ClockSampler:
         self.f.flush()
         self.f.seek(0)
         sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.f.read().splitlines():
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 9:
@@ -140,7 +200,7 @@ class ClockSampler:
                 mx.append(float(parts[2]))
             except ValueError:
                 continue
-            for nm, v in zip(names, parts[5:9]):
+            for nm, v in zip(self.NAMES, parts[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(nm)
         os.unlink(self.f.name)
@@ -243,6 +303,130 @@ def build_layers(lgn, w, specs, tensors, outs):
     return layers
 
 
+class Prepared:
+    """One workload, resident on the device and ready to step."""
+
+    def __init__(self, lgn, name, batch, seed, dev, tensors=None):
+        self.name = name
+        self.w, self.specs = workload_specs(name, batch, seed)
+        w = self.w
+        self.dtype = torch.float32 if w["dtype"] == "f32" else torch.bfloat16
+        self.esize = 4 if w["dtype"] == "f32" else 2
+        self.tensors = tensors if tensors is not None else synth.make_layers(self.specs, self.dtype, str(dev))
+        if w["mode"] == "prune":
+            self.outs = [torch.empty_like(g) for g in self.tensors]
+        else:
+            self.outs = [torch.empty(max(16, lgn.lgn_codes_bytes(g.numel(), w["nbits"])), dtype=torch.uint8, device=dev)
+                         for g in self.tensors]
+        self.layers = build_layers(lgn, w, self.specs, self.tensors, self.outs)
+        self.ws = lgn.new_workspace([g.numel() for g in self.tensors], dev)
+        self.res = lgn.new_results(len(self.tensors), dev)
+        self.total_elems = sum(g.numel() for g in self.tensors)
+        self.bpe = bytes_per_elem(self.esize, w["mode"], w.get("nbits", 6))
+        self.alg_bytes = self.total_elems * self.bpe
+        l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
+        self.flush = None
+        if self.total_elems * self.esize <= 2 * l2_bytes:      # small inputs: flush L2 between timed steps
+            self.flush = torch.empty(max(2 * l2_bytes, 256 << 20), dtype=torch.uint8, device=dev)
+        self.lgn = lgn
+
+    def step(self):
+        self.lgn.lgn_compress_layers(self.layers, self.res, self.ws)
+
+    def warm(self, n):
+        for _ in range(n):
+            if self.flush is not None:
+                self.flush.fill_(1)
+            self.step()
+        torch.cuda.synchronize()
+        status = [r["status"] for r in self.lgn.read_results(self.res, len(self.tensors))]
+        if any(status):
+            raise SystemExit(f"{self.name}: per-layer status not ok: {status}")
+
+    def timed(self, steps):
+        """CUDA-event times of `steps` back-to-back steps on the current stream:
+        (device ms of the whole block, per-step ms list)."""
+        stream = torch.cuda.current_stream()
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        for i in range(steps):
+            if self.flush is not None:
+                self.flush.fill_(1)
+            starts[i].record(stream)
+            self.step()
+            ends[i].record(stream)
+        torch.cuda.synchronize()
+        per = [a.elapsed_time(b) for a, b in zip(starts, ends)]
+        # inputs above L2: the device time of exactly K back-to-back steps; else the flushes
+        # between steps are not part of the path
+        total = starts[0].elapsed_time(ends[-1]) if self.flush is None else sum(per)
+        return total, per
+
+
+# What the counters of one ncu capture say bounds each kind of workload (profiles/): fp32 pruning
+# moves the algorithmic bytes at the HBM rate; the other bodies execute 22-34 instructions per
+# element and sit between the HBM roof and the issue-slot ceiling.
+def roofline_of(name, alg_bytes, per_step_ms):
+    peak, peak_kind = read_peak()
+    kern_ms = statistics.mean(per_step_ms)
+    achieved = alg_bytes / (kern_ms * 1e-3) / 1e9
+    r = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+         "traffic": None, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
+         "kernel": "compress_kernel", "algorithmic_bytes_per_launch": alg_bytes,
+         "best_ms": min(per_step_ms), "median_ms": statistics.median(per_step_ms)}
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            tr = json.load(f).get(name)
+        if tr and tr.get("library_sha") == lib_sha():
+            r["traffic"] = tr["dram_bytes_per_launch"]
+    except Exception:
+        pass
+    try:
+        with open(os.path.join(ROOT, "profiles", "issue_ceilings.json")) as f:
+            ic = json.load(f).get(name)
+        if ic:
+            r["issue_ceiling"] = ic        # instructions per element (ncu) and the GB/s at which every issue slot is used
+    except Exception:
+        pass
+    return r
+
+
+ALSO_DEFAULT = ["resnet18_bs256_fp32_fp6", "resnet50_bs256_bf16_fp6", "resnet50_bs256_bf16_prune",
+                "flat_2p26_fp32_prune", "flat_2p26_fp32_fp6", "flat_2p26_bf16_prune", "flat_2p26_bf16_fp6",
+                "flat_2p30_fp32_prune", "flat_2p30_fp32_fp6", "flat_2p30_bf16_prune", "flat_2p30_bf16_fp6"]
+
+
+def tensor_key(name):
+    w = WORKLOADS[name]
+    return (w["net"], w.get("log2n"), w["dtype"])
+
+
+def run_also(lgn, args, dev, first: "Prepared"):
+    """The other halves of the metric and the other configurations, a few steps each, on the
+    same GPU right after the headline workload: rows of {workload, ms_per_step, value, roofline}."""
+    rows = []
+    names = [n for n in args.also.split(",") if n and n != args.workload]
+    cache_key, cache_tensors = tensor_key(first.name), first.tensors
+    for name in sorted(names, key=lambda n: (tensor_key(n) != cache_key, names.index(n))):
+        if WORKLOADS[name]["net"] == "aux":
+            continue
+        if tensor_key(name) != cache_key:
+            cache_tensors = None
+            torch.cuda.empty_cache()
+        p = Prepared(lgn, name, args.batch, 0, dev, tensors=cache_tensors)
+        cache_key, cache_tensors = tensor_key(name), p.tensors
+        p.warm(3)
+        total_ms, per = p.timed(args.also_steps)
+        ms = total_ms / args.also_steps
+        rows.append({"workload": name, "dtype": p.w["dtype"], "mode": p.w["mode"], "elements": p.total_elems,
+                     "steps": args.also_steps, "ms_per_step": ms, "value": p.alg_bytes / (ms * 1e-3) / 1e9,
+                     "unit": "GB/s", "elements_per_s": p.total_elems / (ms * 1e-3),
+                     "l2": "inputs larger than L2" if p.flush is None else "L2 flushed between timed steps",
+                     "roofline": roofline_of(name, p.alg_bytes, per)})
+        del p
+    return rows
+
+
 def run_ours(args):
     world, rank, local = dist_setup(args.gpus)
     if not torch.cuda.is_available():
@@ -250,99 +434,59 @@ def run_ours(args):
     from paper_2006_08173_b200 import binding as lgn      # raises if liblgn.so is missing
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    w, specs = workload_specs(args.workload, args.batch, rank)
-    dtype = torch.float32 if w["dtype"] == "f32" else torch.bfloat16
-    esize = 4 if w["dtype"] == "f32" else 2
-    tensors = synth.make_layers(specs, dtype, str(dev))
-    if w["mode"] == "prune":
-        outs = [torch.empty_like(g) for g in tensors]
-    else:
-        outs = [torch.empty(max(16, lgn.lgn_codes_bytes(g.numel(), w["nbits"])), dtype=torch.uint8, device=dev)
-                for g in tensors]
-    layers = build_layers(lgn, w, specs, tensors, outs)
-    ws = lgn.new_workspace([g.numel() for g in tensors], dev)
-    res = lgn.new_results(len(tensors), dev)
-    total_elems = sum(g.numel() for g in tensors)
-    bpe = bytes_per_elem(esize, w["mode"], w.get("nbits", 6))
-    alg_bytes = total_elems * bpe
-    in_bytes = total_elems * esize
-    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
-    flush = None
-    if in_bytes <= 2 * l2_bytes:                     # small inputs: flush L2 between timed steps
-        flush = torch.empty(max(2 * l2_bytes, 256 << 20), dtype=torch.uint8, device=dev)
+    P = Prepared(lgn, args.workload, args.batch, rank, dev)
+    w, specs, tensors = P.w, P.specs, P.tensors
 
-    stream = torch.cuda.current_stream()
-    for _ in range(args.warmup):
-        if flush is not None:
-            flush.fill_(1)
-        lgn.lgn_compress_layers(layers, res, ws)
-    torch.cuda.synchronize()
-    status = [r["status"] for r in lgn.read_results(res, len(tensors))]
-    if any(status):
-        raise SystemExit(f"per-layer status not ok: {status}")
-
-    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    sampler = ClockSampler(local) if rank == 0 else None   # runs from before the warm-up to after the load
+    if sampler:
+        sampler.mark("load_begin")
+    P.warm(args.warmup)
     barrier(world)
     torch.cuda.synchronize()
-    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.mark("timed_begin")
     wall0 = time.perf_counter()
-    for i in range(args.steps):
-        if flush is not None:
-            flush.fill_(1)
-        starts[i].record(stream)
-        lgn.lgn_compress_layers(layers, res, ws)
-        ends[i].record(stream)
-    torch.cuda.synchronize()
+    total_ms, per_step_ms = P.timed(args.steps)            # exactly K steps, CUDA events
     wall = time.perf_counter() - wall0
+    if sampler:
+        sampler.mark("timed_end")
     barrier(world)
+    # The timed block can be as short as 20 ms.  The same steps keep running (untimed) until the
+    # GPU has been under this load for half a second, so that the clock record has samples.
+    if sampler:
+        t_hold = time.perf_counter()
+        while time.perf_counter() - sampler.marks["load_begin"] < 0.6 and time.perf_counter() - t_hold < 2.0:
+            P.timed(max(1, min(args.steps, 20)))
+        sampler.mark("load_end")
     clocks = sampler.stop() if sampler else None
-    per_step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
-    if flush is None:
-        total_ms = starts[0].elapsed_time(ends[-1])      # device time of exactly K back-to-back steps
-    else:
-        total_ms = sum(per_step_ms)                      # the flushes between steps are not part of the path
     total_ms = max_over_ranks(total_ms, world, dev)
     ms_per_step = total_ms / args.steps
-    value = world * alg_bytes / (ms_per_step * 1e-3) / 1e9
-
-    peak, peak_kind = read_peak()
-    kern_ms = statistics.mean(per_step_ms)
-    achieved = alg_bytes / (kern_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
-                "kernel": "compress_kernel", "algorithmic_bytes_per_launch": alg_bytes,
-                "best_ms": min(per_step_ms), "median_ms": statistics.median(per_step_ms)}
-    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
-    try:
-        with open(traffic_path) as f:
-            tr = json.load(f).get(args.workload)
-        if tr and tr.get("library_sha") == lib_sha():
-            roofline["traffic"] = tr["dram_bytes_per_launch"]
-    except Exception:
-        pass
+    value = world * P.alg_bytes / (ms_per_step * 1e-3) / 1e9
 
     line = {
         "metric": "fused_stats_apply_algorithmic_GBps", "value": value, "unit": "GB/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": w["dtype"], "data": "synthetic",
-        "config": {"workload": args.workload, "layers": len(tensors), "elements_per_step_per_gpu": total_elems,
+        "config": {"workload": args.workload, "layers": len(tensors), "elements_per_step_per_gpu": P.total_elems,
                    "mode": w["mode"], "nbits": w.get("nbits"), "batch": args.batch,
-                   "l2": "inputs larger than L2" if flush is None else "L2 flushed between timed steps",
+                   "l2": "inputs larger than L2" if P.flush is None else "L2 flushed between timed steps",
                    "parallelism": f"replicas x{world}"},
-        "elements_per_s": world * total_elems / (ms_per_step * 1e-3),
+        "elements_per_s": world * P.total_elems / (ms_per_step * 1e-3),
         "gpu_launches": args.steps * lgn.lgn_launches_per_call(len(tensors)),
-        "roofline": roofline,
+        "roofline": roofline_of(args.workload, P.alg_bytes, per_step_ms),
         "clocks": clocks,
         "wall_s": wall,
     }
 
     if rank == 0 and not args.no_e2e:
-        line["e2e"] = measure_e2e(lgn, args, w, specs, tensors, dev, alg_bytes)
+        line["e2e"] = measure_e2e(lgn, args, w, specs, tensors, dev, P.alg_bytes)
     barrier(world)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = measure_cpu_baseline(args, w, specs, tensors, bpe)
+        line["cpu_baseline"] = measure_cpu_baseline(args, w, specs, tensors, P.bpe)
+        line["cpu_baseline_all_cores"] = measure_cpu_baseline(args, w, specs, tensors, P.bpe, all_cores=True)
+    if rank == 0 and world == 1 and args.also:
+        line["also"] = run_also(lgn, args, dev, P)
     if rank == 0:
         print(json.dumps(line))
 
@@ -511,17 +655,41 @@ def measure_e2e(lgn, args, w, specs, tensors, dev, alg_bytes):
             "pcie_GBps": (h2d + d2h) / dt / 1e9}
 
 
-def measure_cpu_baseline(args, w, specs, tensors, bpe):
+def cpu_model():
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+def measure_cpu_baseline(args, w, specs, tensors, bpe, all_cores=False):
+    """The oracle as it stands on a bounded sample of the workload (its trailing layers): on
+    one thread, or with the layers spread over every core the process may use (threads: the
+    oracle's C functions release the interpreter lock; each layer still runs on one thread)."""
     import oracle as orc
     orc.build()
-    sample, total = oracle_sample(specs, w, args.cpu_sample_elems)
+    cores = len(os.sched_getaffinity(0))
+    budget = args.cpu_sample_elems * (min(cores, 8) if all_cores else 1) // (2 if all_cores else 1)
+    sample, total = oracle_sample(specs, w, budget)
     arrays = [synth.as_numpy_bits(tensors[len(specs) - len(sample) + k]) for k in range(len(sample))]
+    used = 1
     t0 = time.perf_counter()
-    oracle_step(orc, arrays, sample, w)
+    if all_cores:
+        from concurrent.futures import ThreadPoolExecutor
+        used = min(cores, len(sample))
+        order = sorted(range(len(sample)), key=lambda k: -sample[k].numel)     # longest first
+        with ThreadPoolExecutor(used) as ex:
+            list(ex.map(lambda k: oracle_step(orc, [arrays[k]], [sample[k]], w), order))
+    else:
+        oracle_step(orc, arrays, sample, w)
     dt = time.perf_counter() - t0
-    return {"value": total * bpe / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+    return {"value": total * bpe / dt / 1e9, "unit": "GB/s", "cores": used, "kind": "oracle",
             "sample": f"last {len(sample)} of {len(specs)} layers ({total} elements), one pass, {dt:.1f} s",
-            "host_cores_available": len(os.sched_getaffinity(0))}
+            "host_cores_available": cores, "cpu_model": cpu_model()}
 
 
 def main():
@@ -536,6 +704,10 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-elems", type=int, default=300_000_000)
+    ap.add_argument("--also", default=",".join(ALSO_DEFAULT),
+                    help="comma-separated workloads timed after the headline one and reported in the line's `also` list")
+    ap.add_argument("--no-also", action="store_const", const="", dest="also")
+    ap.add_argument("--also-steps", type=int, default=10)
     ap.add_argument("--ref-sample-elems", type=int, default=33_000_000)
     args = ap.parse_args()
     if args.warmup < 3:

@@ -22,8 +22,9 @@
  *  - Tensors are contiguous and are treated as flat arrays of n elements; the
  *    element index used for randomness is the flat index.
  *  - Gradient tensors (g, and out of a pruning call) must be 32-byte aligned;
- *    code streams and workspaces 16-byte aligned, result arrays 8-byte aligned.  Input and
- *    output buffers must not overlap.
+ *    code streams, workspaces and a device lgn_stats_t (lgn_stats,
+ *    lgn_stats_static_scratch) 16-byte aligned, arrays of lgn_layer_result_t 8-byte
+ *    aligned.  Input and output buffers must not overlap.
  *  - Inputs must be finite, with magnitudes below 2^104 (about 2e31).  +0 and -0
  *    both count as zero.
  *  - Argument errors are found on the host and returned before anything is
@@ -57,9 +58,9 @@ typedef enum { LGN_MODE_PRUNE = 0, LGN_MODE_QUANTIZE = 1 } lgn_mode;
  *   LGN_SCALE_CENTRED   e_s = floor(mu/ln 2 + 1/2): the median magnitude sits in the middle
  *                       of the format's range, the setting Eq. 4 is derived for
  *   LGN_SCALE_FROM_MAX  e_s = floor(log2 max|g|) - (E_max - 1): the largest element sits in
- *                       the top binade, nothing is clipped, the smallest elements are given
- *                       up ("sacrifices the smallest elements to keep the largest gradients
- *                       magnitude representable", appendix "Gradient scaling") */
+ *                       the top binade, so nothing is clipped and the range is spent on the
+ *                       large magnitudes at the expense of the smallest ones (the trade
+ *                       described in the appendix "Gradient scaling") */
 typedef enum { LGN_SCALE_CENTRED = 0, LGN_SCALE_FROM_MAX = 1 } lgn_scale_mode;
 
 /* Lognormal statistics of one tensor (Section 3: magnitudes, zeros left out). */
@@ -154,9 +155,9 @@ lgn_status lgn_scale_from_max(double max_abs, int exp_bits, int32_t *scale_exp);
  * heterogeneous stochastic pruning") ----
  * lgn_cosine_similarity: the expected cosine of the angle between a layer's gradient and
  * its stochastically pruned copy at threshold tau, for magnitudes whose logarithm is
- * normal (mu, sigma) and cut off k standard deviations above mu ("the neural gradients'
- * lognormal distributions are truncated"; k is the 0.997 quantile of the data in
- * sigmas, lgn_quantile).  Host only.  tau must be > 0 and ln(tau) - mu <= k*sigma
+ * normal (mu, sigma) and cut off k standard deviations above mu (the appendix observes
+ * that measured gradients lack the lognormal's far upper tail; k is the 0.997 quantile
+ * of the data in sigmas, lgn_quantile).  Host only.  tau must be > 0 and ln(tau) - mu <= k*sigma
  * (a threshold above the cut prunes everything): otherwise LGN_ERR_INVALID_ARG. */
 lgn_status lgn_cosine_similarity(double mu, double sigma, double k, double tau, double *cosine);
 
@@ -189,6 +190,8 @@ lgn_status lgn_allocate_sparsity(const lgn_alloc_layer_t *layers, int num_layers
  *   out_dev  device, 16 bytes, 16-byte aligned: { float value; uint32_t pad; uint64_t nnz }
  *            (value 0 when the tensor has no nonzero element)
  *   ws       device scratch of lgn_quantile_workspace_bytes() bytes, 16-byte aligned
+ * n must be below 2^32 (the histogram bins are 32-bit counters): a larger n returns
+ * LGN_ERR_UNSUPPORTED and nothing is enqueued.
  * Three (bf16) or five (fp32) small launches on `stream`, no allocation. */
 typedef struct { float value; uint32_t pad; uint64_t nnz; } lgn_quantile_t;
 size_t     lgn_quantile_workspace_bytes(void);
@@ -199,11 +202,16 @@ lgn_status lgn_quantile(const void *g, uint64_t n, lgn_dtype dt, double q, lgn_q
  * between refreshes of the statistics.
  *   g, out  device, n elements of dt; out has the same type and layout
  *   tau     alpha >= 0; the kernel uses lgn_snap_threshold(tau, dt)
- *   seed    element i draws eps_i = h_i / 2^16, h_i = 16 bits of a Philox4x32-7
- *           block: key = (seed low, seed high), counter = (i/8 low, i/8 high, 0, 0),
- *           word (i/2) mod 4, low half for even i, high half for odd i
+ *   seed    element i draws eps_i = (h_i + 1) / 2^16 in (0, 1] (Eq. 5's eps ~ U[0,1] on a
+ *           grid of 2^16 points that leaves out 0, so that alpha*eps_i > 0 and a zero can
+ *           never be kept), h_i = 16 bits of a Philox4x32-7 block: key = (seed low, seed
+ *           high), counter = (i/8 low, i/8 high, 0, 0), word (i/2) mod 4, low half for
+ *           even i, high half for odd i
  * |g_i| > alpha -> g_i;  fl32(alpha*eps_i) <= |g_i| <= alpha -> sign(g_i)*alpha;
- * otherwise +0.  Zeros stay +0. */
+ * otherwise +0.  Zeros stay +0.  An element with 0 < |g_i| <= alpha is kept with
+ * probability floor(2^16 |g_i| / alpha) / 2^16 (up to the one rounding of alpha*eps_i),
+ * so E[out_i] falls short of g_i by less than alpha * 2^-16; Eq. 5 with a continuous eps
+ * is exactly unbiased. */
 lgn_status lgn_prune(const void *g, void *out, uint64_t n, lgn_dtype dt, double tau,
                      uint64_t seed, void *stream);
 
@@ -218,7 +226,9 @@ lgn_status lgn_prune(const void *g, void *out, uint64_t n, lgn_dtype dt, double 
  *   E >= E_max  (before rounding) -> largest code;
  *   E <= -E_max (before rounding) -> 0, under both roundings;
  *   else M rounded to man_bits (nearest: ties to the even mantissa; stochastic:
- *   h_i/2^16 of one mantissa step added, then truncated),
+ *   h_i/2^16 of one mantissa step added, then truncated: the value rounds up with
+ *   probability floor(frac * 2^16) / 2^16 for a dropped fraction frac, so the expected
+ *   result falls short of x by less than 2^-16 of one mantissa step),
  *   a carry out of M moves to E, and E reaching E_max gives the largest code.
  * Exponent field = E + E_max (1..2^exp_bits-1); field 0 encodes zero.
  * A code decodes to (-1)^s (1 + m/2^man_bits) 2^(field - E_max + scale_exp). */
@@ -369,7 +379,9 @@ lgn_status lgn_selftest_wait_expires(const lgn_layer_t *layers, int num_layers,
  * The call itself allocates nothing on the device, neither directly nor through
  * a library.  The first call on each device looks up the array's device address
  * (one cudaGetSymbolAddress, with that device current) and remembers it; make
- * that first call before starting any stream capture.
+ * that first call before starting any stream capture.  The look-up is serialised
+ * among host threads, and serves device ordinals 0..63: on a device with a higher
+ * ordinal the call returns LGN_ERR_CUDA and enqueues nothing.
  * All calls on one device share the one array: it still holds the previous
  * call's contents when the next call starts (the call re-initialises what it
  * reads), and two calls whose kernels can overlap on the GPU -- different

@@ -108,7 +108,7 @@ typedef struct {
 
 /* The analysis is done on |g| with the zero entries left out (Section 3);
  * mu and sigma are the mean and standard deviation of the natural log
- * (the "mean and standard deviation of the input", Appendix A.8).
+ * (the two O(n) quantities the method needs, Appendix A.8).
  * Two passes, compensated (Kahan) sums. */
 void orc_stats(const void *g, uint64_t n, int dtype, orc_stats_t *out)
 {
@@ -200,8 +200,8 @@ double orc_max_abs(const void *g, uint64_t n, int dtype)
 
 /* Algorithm 1, the scale from the maximum.  The printed line
  * "mu_l = floor(log2 max|X|) / log2(E_max)" does not give an exponent shift as it
- * stands; the text around it fixes what it is for: the scale "sacrifices the
- * smallest elements to keep the largest gradients magnitude representable".  With
+ * stands; the text around it fixes what it is for: the scale gives up the smallest
+ * elements so that the largest magnitudes stay representable.  With
  * representable exponents -E_max+1 .. E_max-1 that is the power of two that puts
  * the largest element in the top binade:
  *     e_s = floor(log2 max|X|) - (E_max - 1).
@@ -586,7 +586,7 @@ static double Phi(double z) { return 0.5 * erfc(-z / sqrt(2.0)); }
  *
  * Reading: the main text writes the cut as erf((k s - 2 s^2)/(s rt2)), i.e. ln x <= k s,
  * while the step-by-step derivation writes ln(k s) in the same place.  The first is
- * taken: k is "obtained from the distribution like sigma and mu" as a high quantile
+ * taken: k is measured on the data, as mu and sigma are, as a high quantile
  * (0.997: the mass inside three standard deviations of a normal), which is a
  * statement about ln x in units of sigma.  Zeros of the tensor add nothing to any of
  * the three sums.  Requires u <= k s (a threshold above the cut prunes everything).
@@ -640,7 +640,7 @@ static double u_for_sparsity(double Sp, double sigma)
  *   - otherwise it keeps S.
  * The remaining layers share one level that restores the budget,
  *   S_rest = (S * sum_all n_i - sum_deep n_i S_i) / sum_rest n_i,
- * limited to s_max ("a maximum of 0.96-0.98 will prevent over-pruning") and to at
+ * limited to s_max (the appendix recommends a cap of 0.96-0.98 against over-pruning) and to at
  * least S.  out_S[i] receives every layer's sparsity.  Returns the element-weighted
  * mean sparsity actually allocated (below S when the cap binds). */
 double orc_allocate_sparsity(int L, const uint64_t *n, const double *sigma, const double *zero_frac,

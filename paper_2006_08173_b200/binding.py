@@ -14,7 +14,7 @@ from typing import Dict, List, Optional, Sequence
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("LGN_LIBRARY", os.path.join(_PKG, "liblgn.so"))   # override: another build of the same ABI
+LIB_PATH = os.path.join(_PKG, "liblgn.so")      # the in-tree build, and nothing else
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(

@@ -19,7 +19,7 @@ _DEPS = SOURCES + [os.path.join(_CSRC, "lgn_device.cuh"), os.path.join(_CSRC, "l
 def nvcc_command(extra=()):
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     return [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(_ROOT, "include"), "-I", _CSRC,
+            "--threads", "0", "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(_ROOT, "include"), "-I", _CSRC,
             *extra, "-o", LIB_PATH, *SOURCES]
 
 

@@ -16,6 +16,7 @@
 // tiles in the queue, so every wait is on work already handed to a running CTA.
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include <cuda_runtime.h>
@@ -359,6 +360,12 @@ __device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn *D, co
         *L.result_out = r;
     }
     __threadfence();
+    // A waiter that gave up on this layer before now has skipped tiles: its verdict
+    // stands, whichever of the two stores to the record's status lands first.
+    if (atomicAdd(&D->status, 0) != 0 && L.result_out) {
+        *(volatile int32_t *)&L.result_out->status = LGN_ERR_TIMEOUT;
+        __threadfence();
+    }
     st_release(&D->ready, 1u);
 }
 
@@ -456,13 +463,17 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
         } else {
             if ((int)sg.layer != ready_layer) {
                 if (threadIdx.x == 0) {
+                    // The wait is this layer's own: it ends early only when another waiter of
+                    // the SAME layer has already given up.  Layers whose statistics are merely
+                    // still running keep their full count whatever happened elsewhere.
                     uint32_t polls = 0, ok = 1;
                     while (ld_acquire(&D->ready) == 0u) {
-                        if (++polls > kMaxPolls || *(volatile uint32_t *)&hdr->error) { ok = 0; break; }
+                        if (++polls > kMaxPolls || *(volatile int32_t *)&D->status != 0) { ok = 0; break; }
                         __nanosleep(100);
                     }
                     if (!ok) {
-                        atomicExch(&hdr->error, 1u);
+                        if (atomicCAS(&D->status, 0, (int32_t)LGN_ERR_TIMEOUT) == 0) atomicExch(&hdr->error, 1u);
+                        __threadfence();                           // after a record finalize_layer may have stored
                         if (L.result_out) *(volatile int32_t *)&L.result_out->status = LGN_ERR_TIMEOUT;
                     }
                     sm_flag = ok;
@@ -1032,11 +1043,14 @@ extern "C" lgn_status lgn_selftest_wait_expires(const lgn_layer_t *layers, int n
 static __device__ __align__(256) unsigned char g_stats_static_scratch[LGN_STATS_STATIC_SCRATCH_BYTES];
 
 namespace {
-// Device address of the array on the current device, looked up once per device.
+// Device address of the array on the current device, looked up once per device
+// (ordinals 0..63; host threads that make the first call together take turns).
 void *static_scratch_address() {
     static void *cached[64];
+    static std::mutex guard;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(guard);
     if (cached[dev] == nullptr) {
         void *p = nullptr;
         if (cudaGetSymbolAddress(&p, g_stats_static_scratch) != cudaSuccess) return nullptr;

@@ -1,7 +1,7 @@
 // Exact order statistic of |g| over the nonzero elements (the high quantile that
 // estimates the cut k of a truncated lognormal; appendix "Neural gradients lognormal
-// distributions are truncated": "in practice we take a high quantile (for example
-// 0.997) of the distribution").
+// distributions are truncated", which takes a high quantile of the data, 0.997 as its
+// example, for the cut).
 //
 // Magnitude patterns of IEEE values order like the values, so the element of rank r
 // is found by radix selection on the pattern:
@@ -192,7 +192,7 @@ extern "C" lgn_status lgn_quantile(const void *g, uint64_t n, lgn_dtype dt, doub
     if (!(q >= 0.0 && q <= 1.0)) return LGN_ERR_INVALID_ARG;
     if (out_dev == nullptr || (reinterpret_cast<uintptr_t>(out_dev) & 15u)) return LGN_ERR_INVALID_ARG;
     if (n > 0 && (g == nullptr || (reinterpret_cast<uintptr_t>(g) & 31u))) return LGN_ERR_INVALID_ARG;
-    if (n > (1ull << 44)) return LGN_ERR_UNSUPPORTED;
+    if (n >= (1ull << 32)) return LGN_ERR_UNSUPPORTED;       // the histogram bins count in 32 bits
     if (ws == nullptr || (reinterpret_cast<uintptr_t>(ws) & 15u)) return LGN_ERR_INVALID_ARG;
     if (ws_bytes < kQWsBytes) return LGN_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -1,5 +1,8 @@
 """Shared helpers of the GPU parity tests: run the oracle for one layer and
 compare the library's outputs with it."""
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import torch
 
@@ -10,6 +13,40 @@ REL_TOL = 1e-5      # mu / sigma: relative to the oracle's fp64 value
 
 def np_bits(t):
     return synth.as_numpy_bits(t).reshape(-1)
+
+
+# The oracle's C functions release the interpreter lock: host threads run it in parallel.
+THREADS = max(1, len(os.sched_getaffinity(0)))
+
+
+def on_threads(fn, jobs):
+    with ThreadPoolExecutor(THREADS) as ex:
+        return list(ex.map(lambda j: fn(*j), jobs))
+
+
+def oracle_stats_whole(oracle, tensors):
+    """oracle.stats of every tensor over all of its elements, one tensor at a time on the
+    host (a device tensor is copied, measured, and its host copy dropped)."""
+    def one(g):
+        return oracle.stats(np_bits(g))
+    return on_threads(one, [(g,) for g in tensors])
+
+
+def windows_of(n, tile, rs, width=65536, seams=3, rand=3, full_below=3_000_000):
+    """Windows [lo, hi) of a tensor of n elements: the whole tensor when small; else its
+    first and last `width` elements, windows straddling tile seams (at the start, in the
+    middle and near the end of the tensor) and random ones.  Starts are multiples of 8."""
+    if n <= full_below:
+        return [(0, n)]
+    w = [(0, width), (n - width - (n - width) % 8, n)]
+    ntiles = n // tile
+    for k in sorted(set([1, ntiles // 2, max(1, ntiles - 1)]))[:seams]:
+        lo = k * tile - width // 2
+        if 0 <= lo and lo + width <= n:
+            w.append((lo, lo + width))
+    for x in rs.randint(0, (n - width) // 8, rand):
+        w.append((int(x) * 8, int(x) * 8 + width))
+    return w
 
 
 def oracle_layer(orc, g_np, mode, *, S=0.0, nbits=6, rounding=0, seed=0):

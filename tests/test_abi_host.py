@@ -165,6 +165,20 @@ def test_device_entry_points_reject_bad_arguments_before_any_cuda_call(lgn):
     assert call(layer(), n=0) == 0
 
 
+def test_quantile_rejects_bad_arguments_before_any_cuda_call(lgn):
+    R = lgn.raw()
+    A, O, W = 0x10000, 0x90000, 0x200000
+    need = lgn.lgn_quantile_workspace_bytes()
+    INVALID, UNSUPPORTED, WORKSPACE = 1, 2, 3
+    assert R.lgn_quantile(A, 100, 0, 1.5, O, W, need, None) == INVALID
+    assert R.lgn_quantile(A + 8, 100, 0, 0.5, O, W, need, None) == INVALID
+    assert R.lgn_quantile(A, 100, 0, 0.5, O + 8, W, need, None) == INVALID
+    assert R.lgn_quantile(A, 100, 0, 0.5, O, W, need - 1, None) == WORKSPACE
+    # the bins are 32-bit counters: a tensor that could overflow one is refused
+    assert R.lgn_quantile(A, 2 ** 32, 1, 0.5, O, W, need, None) == UNSUPPORTED
+    assert R.lgn_quantile(A, 2 ** 40, 0, 0.5, O, W, need, None) == UNSUPPORTED
+
+
 def test_dequantize_rejects_bad_arguments_before_any_cuda_call(lgn):
     R = lgn.raw()
     A, B = 0x10000, 0x90000

@@ -45,3 +45,33 @@ def test_wait_runs_out_and_is_reported(lgn, oracle):
     assert r2[0]["status"] == 0 and r2[1]["status"] == 0
     assert torch.equal(ob, ob2)
     assert abs(float((oa2 == 0).float().mean()) - 0.8) < 5e-3
+
+
+def test_a_time_out_stays_with_its_own_layer(lgn):
+    """Four layers; layer 0 never completes.  Layer 1 is large enough (120 MB) for the
+    queue to place the statistics of layers 2 and 3 behind layer 0's apply tiles, so they
+    are still to run when layer 0's waiters give up: they, and layer 1, must come back
+    LGN_OK and bit for bit what a normal call writes."""
+    sizes = [1_000_000, 30_000_000, 8_000_000, 8_000_003]
+    gs = [synth.lognormal_tensor(n, -12.0 + k, 2.0, 0.4, seed=40 + k, device="cuda") for k, n in enumerate(sizes)]
+    S = [0.8, 0.7, 0.9, 0.85]
+
+    def run(call):
+        outs = [torch.full_like(g, 7.0) for g in gs]
+        layers = [lgn.make_layer(g, o, lgn.MODE_PRUNE, S=s, seed=10 + k) for k, (g, o, s) in enumerate(zip(gs, outs, S))]
+        ws = lgn.new_workspace(sizes, "cuda")
+        res = lgn.new_results(len(gs), "cuda")
+        call(layers, res, ws)
+        torch.cuda.synchronize()
+        return outs, lgn.read_results(res, len(gs))
+
+    good_out, good = run(lgn.lgn_compress_layers)
+    assert all(r["status"] == 0 for r in good)
+    t0 = time.time()
+    outs, r = run(lgn.lgn_selftest_wait_expires)
+    assert time.time() - t0 < 30.0
+    assert r[0]["status"] == 5 and bool((outs[0] == 7.0).all())
+    for k in (1, 2, 3):
+        assert r[k]["status"] == 0, k
+        assert r[k] == good[k]
+        assert torch.equal(outs[k].view(torch.int32), good_out[k].view(torch.int32)), k

@@ -10,7 +10,7 @@ import pytest
 import torch
 
 import bench
-from gpu_helpers import assert_stats_close, np_bits
+from gpu_helpers import assert_stats_close, np_bits, on_threads, windows_of
 from paper_2006_08173_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -68,15 +68,15 @@ def test_bench_workload_full_size(lgn, oracle):
         tau = oracle.snap_tau(oracle.threshold(st["mu"], st["sigma"], st["zero_frac"], s.sparsity), oracle.F32)
         assert r["tau"] == tau
         n = g.numel()
-        if n <= 7_000_000:
-            windows = [(0, n)]                                                    # the small layers in full
-        else:
-            windows = [(0, 40_000), (n - 40_000, n)] + \
-                      [(int(x), int(x) + 40_000) for x in rs.randint(0, n - 40_000, 3)]
-        for lo, hi in windows:
+        # the small layers in full; about 3.5 M elements of every other layer: its first and
+        # last half million, windows across tile seams and random ones
+        windows = windows_of(n, 32768, rs, width=1 << 19, full_below=7_000_000)
+
+        def one(lo, hi, g=g, o=o, tau=tau, k=k):
             ref = oracle.prune(np_bits(g[lo:hi]), tau, 1000 + k, first=lo)
-            got = np_bits(o[lo:hi])
-            assert np.array_equal(got.view(np.uint32), ref.view(np.uint32)), (k, lo)
+            return np.array_equal(np_bits(o[lo:hi]).view(np.uint32), ref.view(np.uint32))
+        for (lo, hi), ok in zip(windows, on_threads(one, windows)):
+            assert ok, (k, lo, hi)
 
 
 @pytest.mark.parametrize("mode", ["quant", "prune"])

@@ -121,6 +121,33 @@ def test_prune_threshold_product_is_rounded_to_fp32(oracle):
     assert oracle.prune_one(below, tau, h) == 0.0
 
 
+def test_prune_keep_probability_enumerated_over_all_draws(oracle):
+    """Eq. 5 on the grid eps = (h+1)/2^16: over all 2^16 values of h an element with
+    0 < |x| <= alpha is kept exactly floor(2^16 |x| / alpha) times (alpha a power of two, so
+    alpha*eps is exact), hence E[T(x)] = alpha * floor(2^16 |x|/alpha) / 2^16 lies in
+    (|x| - alpha 2^-16, |x|]: the bias of the 16-bit grid, against the exact unbiasedness
+    of a continuous eps.  For a full-mantissa alpha the one fp32 rounding of alpha*eps can
+    move the count by at most one."""
+    hs = np.arange(1 << 16, dtype=np.uint16)
+    for alpha in (1.0, 2.0 ** -14, 2.0 ** 10):
+        for ratio in (2.0 ** -16, 3 * 2.0 ** -16, 0.1, 1 / 3, 0.5, 0.75 - 2.0 ** -20, 0.999, 1.0):
+            x = float(np.float32(alpha * ratio))
+            g = np.full(1 << 16, -x, dtype=np.float32)
+            out = oracle.prune_with_bits(g, alpha, hs)
+            kept = int(np.count_nonzero(out))
+            assert kept == math.floor((1 << 16) * (x / alpha)), (alpha, ratio)
+            assert np.all(out[out != 0] == np.float32(-alpha))
+            mean = -float(out.astype(np.float64).mean())
+            assert x - alpha * 2.0 ** -16 < mean <= x
+        below = float(np.float32(alpha * 2.0 ** -17))                   # under the smallest alpha*eps: never kept
+        assert np.count_nonzero(oracle.prune_with_bits(np.full(1 << 16, below, dtype=np.float32), alpha, hs)) == 0
+    alpha = float(np.float32(1.2345678))
+    for ratio in (0.1, 0.37, 0.9):
+        x = float(np.float32(alpha * ratio))
+        kept = int(np.count_nonzero(oracle.prune_with_bits(np.full(1 << 16, x, dtype=np.float32), alpha, hs)))
+        assert abs(kept - (1 << 16) * x / alpha) <= 1.0 + 1e-9
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_prune_three_value_property(oracle, dtype):
     n = 200_000

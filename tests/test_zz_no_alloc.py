@@ -37,6 +37,26 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(lgn, oracle):
     assert got == ref and got["n"] == 0
 
 
+def test_the_call_leaves_free_device_memory_as_it_found_it(lgn):
+    """The one promise of this entry point: nothing is allocated.  Everything the test
+    itself needs exists before the first reading of cudaMemGetInfo; the first call (which
+    looks the array's address up) has been made; the second call must leave the free
+    byte count where it was."""
+    g = synth.lognormal_tensor(2_000_003, -11.0, 2.0, 0.3, seed=25, device="cuda")
+    out = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    lgn.lgn_stats_static_scratch_async(g, out)
+    torch.cuda.synchronize()
+    first = lgn.read_stats(out)
+    out.zero_()
+    torch.cuda.synchronize()
+    free_before, total = torch.cuda.mem_get_info()
+    lgn.lgn_stats_static_scratch_async(g, out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    assert lgn.read_stats(out) == first
+
+
 def test_back_to_back_without_a_sync_between_them(lgn):
     a = synth.lognormal_tensor(1_000_000, -12.0, 2.0, 0.5, seed=23, device="cuda")
     b = synth.lognormal_tensor(500_000, -6.0, 1.5, 0.0, seed=24, device="cuda")
