@@ -123,7 +123,7 @@ static bool ws_layout(const uint64_t *n_per_layer, int L, WsLayout &w) {
 // (more than a dozen layers) in launches of kBigBlobBytes each, so that a call with
 // a hundred layers still has a single set-up launch.
 constexpr int kBlobBytes = 3840;
-constexpr int kBigBlobBytes = 30720;
+constexpr int kBigBlobBytes = 32512;
 template <int BYTES> struct BlobT { uint4 v[BYTES / 16]; };
 
 template <int BYTES>
@@ -379,7 +379,7 @@ __device__ __forceinline__ QuantParams load_quant_params(const LayerDyn *D) {
 }
 
 // ------------------------------------------------------------------ the persistent kernel
-constexpr uint32_t kMaxPolls = 1u << 20;      // x ~1 us per poll (acquire load + back-off): about one second
+constexpr uint32_t kMaxPolls = 1u << 19;      // x ~1 us per poll (acquire load + back-off): about half a second
 constexpr int kAny = -1;                      // template value: decided per layer at run time
 
 // DT, MODE, NBITS, SR fix what every layer of the group has in common, so that
@@ -466,9 +466,20 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
                     // The wait is this layer's own: it ends early only when another waiter of
                     // the SAME layer has already given up.  Layers whose statistics are merely
                     // still running keep their full count whatever happened elsewhere.
-                    uint32_t polls = 0, ok = 1;
+                    // The count starts again whenever the queue has moved: the statistics tile
+                    // this wait depends on may be in the hands of a CTA that is itself sitting
+                    // out the wait of a layer that will never complete, and resumes after it.
+                    // Such a CTA holds items that lie LATER in the queue than the one it waits
+                    // for, so patience grows with the layer's position: the waiters of an
+                    // earlier layer always give up, and move on, first.
+                    const uint32_t limit = kMaxPolls * (1u + (sg.layer < 15u ? sg.layer : 15u));
+                    uint32_t polls = 0, ok = 1, seen = *(volatile uint32_t *)&hdr->queue_head;
                     while (ld_acquire(&D->ready) == 0u) {
-                        if (++polls > kMaxPolls || *(volatile int32_t *)&D->status != 0) { ok = 0; break; }
+                        if (++polls > limit || *(volatile int32_t *)&D->status != 0) { ok = 0; break; }
+                        if ((polls & 1023u) == 0u) {
+                            const uint32_t head = *(volatile uint32_t *)&hdr->queue_head;
+                            if (head != seen) { seen = head; polls = 0u; }
+                        }
                         __nanosleep(100);
                     }
                     if (!ok) {

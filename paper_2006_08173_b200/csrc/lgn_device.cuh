@@ -36,6 +36,14 @@ constexpr int kWarps     = kThreads / 32;
 constexpr int kTileElems = LGN_TILE_ELEMS;
 constexpr int kMinCtas   = LGN_MIN_CTAS;      // resident CTAs per SM the kernels are compiled for
 constexpr int kInFlight  = LGN_LOADS_IN_FLIGHT;   // 32-byte loads a thread issues before it uses the first
+#ifndef LGN_PREFETCH_STEPS
+#define LGN_PREFETCH_STEPS 4
+#endif
+// Load steps of a whole tile that are requested into L2 ahead of the register loads (0: none).  A
+// thread holds only one or two 32-byte loads in registers; the lines of the next few steps are
+// asked for with prefetch.global.L2 (no register, no wait), so that the register load that
+// follows finds them in L2.  Four steps (32 KiB per CTA) is the measured optimum.
+constexpr int kPrefetchSteps = LGN_PREFETCH_STEPS;
 
 template <int DT> struct ElemTraits;
 template <> struct ElemTraits<LGN_F32>  { static constexpr int kChunk = 8;  static constexpr int kBytes = 4; };
@@ -148,11 +156,25 @@ __device__ __forceinline__ void pipelined_tile(const void *g, uint64_t tile_base
     constexpr int C = ElemTraits<DT>::kChunk;
     static_assert(kLoads % (2 * kGroup) == 0, "load steps come in pairs of groups");
     Chunk a[kGroup], b[kGroup];
+    // this thread's chunk of load step 0; step j lies j * kStepBytes further on
+    const char *mine = static_cast<const char *>(g) + (tile_base + (uint64_t)threadIdx.x * C) * ElemTraits<DT>::kBytes;
+    constexpr int kStepBytes = kThreads * 32;
+    if (FULL && kPrefetchSteps > 0) {
+        #pragma unroll
+        for (int j = kGroup; j < kGroup + kPrefetchSteps && j < kLoads; ++j)
+            asm volatile("prefetch.global.L2 [%0];" :: "l"(mine + (size_t)j * kStepBytes));
+    }
     #pragma unroll
     for (int j = 0; j < kGroup; ++j)
         a[j] = load_chunk<DT, FULL, P>(g, tile_base + (uint64_t)(j * kThreads + threadIdx.x) * C, n);
     #pragma unroll 1
     for (int j0 = 0; j0 < kLoads; j0 += 2 * kGroup) {
+        if (FULL && kPrefetchSteps > 0) {
+            #pragma unroll
+            for (int j = 0; j < 2 * kGroup; ++j)
+                if (j0 + kGroup + kPrefetchSteps + j < kLoads)
+                    asm volatile("prefetch.global.L2 [%0];" :: "l"(mine + (size_t)(j0 + kGroup + kPrefetchSteps + j) * kStepBytes));
+        }
         #pragma unroll
         for (int j = 0; j < kGroup; ++j)
             b[j] = load_chunk<DT, FULL, P>(g, tile_base + (uint64_t)((j0 + kGroup + j) * kThreads + threadIdx.x) * C, n);
@@ -195,6 +217,37 @@ __device__ __forceinline__ uint4 rand_block(uint64_t seed, uint64_t b, const Wey
         c2 = n2;
     }
     return make_uint4(c0, c1, c2, c3);
+}
+
+// Blocks b and b + 1 for an even b (the 16 elements of a bf16 chunk), rounds interleaved so
+// that each round key is formed once for both.
+__device__ __forceinline__ void rand_block2(uint64_t seed, uint64_t b, const Weyl &wy, uint4 &ra, uint4 &rb) {
+    uint32_t a0 = (uint32_t)b, a1 = (uint32_t)(b >> 32), a2 = 0u, a3 = 0u;
+    uint32_t b0 = a0 + 1u, b1 = a1, b2 = 0u, b3 = 0u;       // b is even: no carry into the second word
+    const uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+    #pragma unroll
+    for (int r = 0; r < kPhiloxRounds; ++r) {
+        const uint32_t key0 = k0 + (uint32_t)r * wy.w0, key1 = k1 + (uint32_t)r * wy.w1;
+        const unsigned long long p0 = (unsigned long long)0xD2511F53u * a0, p1 = (unsigned long long)0xCD9E8D57u * a2;
+        const unsigned long long q0 = (unsigned long long)0xD2511F53u * b0, q1 = (unsigned long long)0xCD9E8D57u * b2;
+        const uint32_t na0 = (uint32_t)(p1 >> 32) ^ a1 ^ key0, na2 = (uint32_t)(p0 >> 32) ^ a3 ^ key1;
+        const uint32_t nb0 = (uint32_t)(q1 >> 32) ^ b1 ^ key0, nb2 = (uint32_t)(q0 >> 32) ^ b3 ^ key1;
+        a1 = (uint32_t)p1; a3 = (uint32_t)p0; a0 = na0; a2 = na2;
+        b1 = (uint32_t)q1; b3 = (uint32_t)q0; b0 = nb0; b2 = nb2;
+    }
+    ra = make_uint4(a0, a1, a2, a3);
+    rb = make_uint4(b0, b1, b2, b3);
+}
+
+// The C/8 blocks of the chunk that starts at element i.
+template <int DT, bool FULL>
+__device__ __forceinline__ void rand_chunk(uint64_t seed, uint64_t i, const Weyl &wy, uint4 (&rr)[ElemTraits<DT>::kChunk / 8]) {
+    if constexpr (DT == LGN_BF16 && FULL) {
+        rand_block2(seed, i >> 3, wy, rr[0], rr[1]);
+    } else {
+        #pragma unroll
+        for (int b = 0; b < ElemTraits<DT>::kChunk / 8; ++b) rr[b] = rand_block(seed, (i >> 3) + b, wy);
+    }
 }
 
 __device__ __forceinline__ uint32_t rand_word(const uint4 &r, int e) {
@@ -252,6 +305,40 @@ __device__ __forceinline__ void stats_tile(const void *g, uint64_t tile_base, ui
     constexpr int kGroup = 16 / C;                        // chunks per register buffer (two buffers): one run of 16
     const float kUnset = -__int_as_float(0x7F800000);     // -inf: no nonzero seen yet
     float P = kUnset;
+    if constexpr (FULL && DT == LGN_BF16) {
+        // Whole bf16 tiles (the pass is bound by instruction issue there; on fp32 tiles, which wait
+        // for memory, this form measured 1 % slower): the thread's 128 (or 256) pivoted terms of
+        // the tile are summed in fp32 (they are of the order of the spread, a sum of squares stays
+        // far below 2^24 ulps) and go to fp64 once per tile; the pivot is fixed by the first group
+        // of 16 that holds a nonzero.
+        float s1 = 0.f, s2 = 0.f, cf = 0.f;
+        pipelined_tile<DT, FULL, Ld::Keep, kLoads, kGroup>(g, tile_base, n, [&](const Chunk (&v)[kGroup], int) {
+            float y[kGroup * C];
+            #pragma unroll
+            for (int idx = 0; idx < kGroup * C; ++idx)
+                y[idx] = lg2_scaled(fabsf(u2f(elem_bits<DT>(v[idx / C], idx % C))));      // -inf for zero
+            if (P == kUnset) {
+                #pragma unroll
+                for (int idx = 0; idx < kGroup * C; ++idx) P = fmaxf(P, y[idx]);
+            }
+            #pragma unroll
+            for (int idx = 0; idx < kGroup * C; ++idx) {
+                if (y[idx] != kUnset) {                    // predicated: no select, no integer add
+                    const float d = y[idx] - P;
+                    s1 += d;
+                    s2 = fmaf(d, d, s2);
+                    cf += 1.0f;                            // exact: at most 256 per tile
+                }
+            }
+        });
+        if (cf != 0.f) {
+            const double p = (double)P - (double)kLogShift, c = (double)cf, D1 = (double)s1, D2 = (double)s2;
+            acc.s1 += D1 + c * p;
+            acc.s2 += D2 + p * (2.0 * D1 + c * p);
+            acc.cnt += (unsigned long long)cf;
+        }
+        return;
+    }
     double D1 = 0.0, D2 = 0.0;
     unsigned long long Cn = 0;
     pipelined_tile<DT, FULL, Ld::Keep, kLoads, kGroup>(g, tile_base, n, [&](const Chunk (&v)[kGroup], int) {
@@ -467,9 +554,11 @@ __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t ti
             if (tau == 0.f) {
                 o = v[j];                                  // alpha = 0: the tensor is left as it is
             } else {
+                uint4 rr[C / 8];
+                rand_chunk<DT, FULL>(seed, i, wy, rr);
                 #pragma unroll
                 for (int b = 0; b < C / 8; ++b) {
-                    const uint4 r = rand_block(seed, (i >> 3) + b, wy);
+                    const uint4 r = rr[b];
                     if constexpr (FULL && DT == LGN_BF16) {
                         const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
                         #pragma unroll
@@ -675,10 +764,13 @@ __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint6
             uint32_t cw[NW + 1];
             #pragma unroll
             for (int k = 0; k <= NW; ++k) cw[k] = 0u;
+            uint4 rr[C / 8];
+            #pragma unroll
+            for (int b = 0; b < C / 8; ++b) rr[b] = make_uint4(0u, 0u, 0u, 0u);
+            if (SR) rand_chunk<DT, FULL>(seed, i, wy, rr);
             #pragma unroll
             for (int b = 0; b < C / 8; ++b) {
-                uint4 r = make_uint4(0u, 0u, 0u, 0u);
-                if (SR) r = rand_block(seed, (i >> 3) + b, wy);
+                const uint4 r = rr[b];
                 if constexpr (DT == LGN_BF16 && FAST) {
                     const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
                     #pragma unroll
