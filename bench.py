@@ -613,7 +613,7 @@ def run_aux(args):
 def lib_sha():
     import hashlib
     h = hashlib.sha1()
-    for rel in ("paper_2006_08173_b200/csrc/lgn.cu", "paper_2006_08173_b200/csrc/lgn_device.cuh",
+    for rel in ("paper_2006_08173_b200/csrc/lgn.cu", "paper_2006_08173_b200/csrc/lgn_kernels.cuh", "paper_2006_08173_b200/csrc/lgn_device.cuh",
                 "paper_2006_08173_b200/csrc/lgn_closed_form.cuh"):
         with open(os.path.join(ROOT, rel), "rb") as f:
             h.update(f.read())
