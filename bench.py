@@ -649,7 +649,7 @@ def measure_e2e(lgn, args, w, specs, tensors, dev, alg_bytes):
         lgn.lgn_compress_layers_host(layers, dev_buf)      # returns after the stream has drained
     dt = (time.perf_counter() - t0) / args.e2e_steps
     h2d = sum(h.numel() * h.element_size() for h in host_in)
-    d2h = sum(h.numel() * h.element_size() for h in host_out) + 88 * len(layers)
+    d2h = sum(h.numel() * h.element_size() for h in host_out) + 120 * len(layers)
     return {"value": alg_bytes / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
             "ms_per_step": dt * 1e3, "steps": args.e2e_steps,
             "pcie_GBps": (h2d + d2h) / dt / 1e9}

@@ -260,6 +260,15 @@ typedef struct {
      * (step 3), S' = (S - l)/(1 - l) (step 2), and the threshold so obtained prunes the
      * WHOLE tensor (step 4). */
     const void  *right_mode;
+    /* Nonzero: the apply pass also counts what it did to this layer (n_zero_out .. n_underflow
+     * of the result record).  The counts cost the integer pipe a few instructions per element
+     * (measured on B200: a call takes 10 % (fp32 FP6) to 30 % (bf16 pruning) longer), so they
+     * are taken only by a second set of kernels, the one
+     * that also serves right_mode and LGN_SCALE_FROM_MAX: a call runs through it, and every
+     * layer of the call then gets its counts, as soon as one layer asks for any of the three,
+     * and so does every call whose layers differ in type, mode, width or rounding. */
+    int32_t      counters;
+    int32_t      reserved;   /* 0 */
 } lgn_layer_t;
 
 typedef struct {
@@ -271,6 +280,14 @@ typedef struct {
     float            max_abs; /* max|g| over the whole tensor; measured only for layers     */
                               /* with LGN_SCALE_FROM_MAX or a right_mode mask, else 0       */
     uint64_t         n_right_mode;  /* with a mask: entries whose mask byte != 0; else 0   */
+    /* What the apply pass did (see lgn_layer_t.counters; all 0 when the call did not count):  */
+    uint64_t         n_zero_out;    /* prune: output elements that are zero (achieved sparsity  */
+                                    /* = n_zero_out / n); quantize: codes that are zero         */
+    uint64_t         n_snapped;     /* prune: elements set to +-alpha (Eq. 5, middle case)      */
+    uint64_t         n_saturated;   /* quantize: codes of the largest magnitude, where values    */
+                                    /* at or beyond the top of the range land (Eq. 2, clip)      */
+    uint64_t         n_underflow;   /* quantize: nonzero elements below the smallest normal,     */
+                                    /* flushed to the zero code (Eq. 2, E <= -E_max)             */
 } lgn_layer_result_t;
 
 /* The whole path for a list of tensors in one kernel launch (plus one tiny

@@ -53,15 +53,18 @@ class LayerT(C.Structure):
                 ("dt", C.c_int32), ("mode", C.c_int32), ("S", C.c_double),
                 ("nbits", C.c_int32), ("rounding", C.c_int32), ("seed", C.c_uint64),
                 ("use_override", C.c_int32), ("scale_mode", C.c_int32),
-                ("mu_override", C.c_double), ("sigma_override", C.c_double), ("right_mode", C.c_void_p)]
+                ("mu_override", C.c_double), ("sigma_override", C.c_double), ("right_mode", C.c_void_p),
+                ("counters", C.c_int32), ("reserved", C.c_int32)]
 
 
 class LayerResultT(C.Structure):
     _fields_ = [("stats", StatsT), ("tau", C.c_double), ("fmt", FpFormatT),
-                ("status", C.c_int32), ("max_abs", C.c_float), ("n_right_mode", C.c_uint64)]
+                ("status", C.c_int32), ("max_abs", C.c_float), ("n_right_mode", C.c_uint64),
+                ("n_zero_out", C.c_uint64), ("n_snapped", C.c_uint64), ("n_saturated", C.c_uint64),
+                ("n_underflow", C.c_uint64)]
 
 
-assert C.sizeof(StatsT) == 48 and C.sizeof(LayerT) == 88 and C.sizeof(LayerResultT) == 88
+assert C.sizeof(StatsT) == 48 and C.sizeof(LayerT) == 96 and C.sizeof(LayerResultT) == 120
 
 _vp, _u64, _sz, _dbl, _i32 = C.c_void_p, C.c_uint64, C.c_size_t, C.c_double, C.c_int
 _lib.lgn_status_string.argtypes = [_i32]
@@ -309,8 +312,9 @@ def lgn_dequantize(codes: torch.Tensor, n: int, fmt: Dict[str, int], out: torch.
 def make_layer(g: torch.Tensor, out: torch.Tensor, mode: int, S: float = 0.0, nbits: int = 0,
                rounding: int = ROUND_NEAREST, seed: int = 0, mu_override: Optional[float] = None,
                sigma_override: Optional[float] = None, scale_mode: int = SCALE_CENTRED,
-               right_mode: Optional[torch.Tensor] = None) -> LayerT:
-    """``right_mode``: uint8/bool CUDA tensor of g.numel() bytes (bi-modal pruning), or None."""
+               right_mode: Optional[torch.Tensor] = None, counters: bool = False) -> LayerT:
+    """``right_mode``: uint8/bool CUDA tensor of g.numel() bytes (bi-modal pruning), or None.
+    ``counters``: have the apply pass fill n_zero_out .. n_underflow of the layer's result."""
     use = mu_override is not None and sigma_override is not None
     mask = None
     if right_mode is not None:
@@ -320,13 +324,14 @@ def make_layer(g: torch.Tensor, out: torch.Tensor, mode: int, S: float = 0.0, nb
     return LayerT(_dev(g, "g") if g.numel() else (g.data_ptr() or None),
                   _dev(out, "out") if out.numel() else (out.data_ptr() or None), g.numel(), dtype_code(g),
                   mode, float(S), int(nbits), int(rounding), int(seed), 1 if use else 0, int(scale_mode),
-                  float(mu_override) if use else 0.0, float(sigma_override) if use else 0.0, mask)
+                  float(mu_override) if use else 0.0, float(sigma_override) if use else 0.0, mask,
+                  1 if counters else 0, 0)
 
 
 def lgn_compress_layers(layers: Sequence[LayerT], results_dev: torch.Tensor, ws: torch.Tensor,
                         stream=None) -> None:
     """Enqueue the grouped path.  ``results_dev``: uint8 CUDA tensor of at least
-    88 bytes per layer; ``ws``: uint8 CUDA tensor of lgn_workspace_bytes(...)."""
+    120 bytes per layer; ``ws``: uint8 CUDA tensor of lgn_workspace_bytes(...)."""
     L = len(layers)
     arr = (LayerT * max(1, L))(*layers)
     if results_dev.numel() * results_dev.element_size() < L * C.sizeof(LayerResultT):
@@ -360,7 +365,9 @@ def read_results(results_dev: torch.Tensor, num_layers: int) -> List[Dict]:
                     "mu": r.stats.mu, "sigma": r.stats.sigma, "tau": r.tau,
                     "fmt": {"nbits": r.fmt.nbits, "exp_bits": r.fmt.exp_bits, "man_bits": r.fmt.man_bits,
                             "scale_exp": r.fmt.scale_exp},
-                    "status": r.status, "max_abs": r.max_abs, "n_right_mode": r.n_right_mode})
+                    "status": r.status, "max_abs": r.max_abs, "n_right_mode": r.n_right_mode,
+                    "n_zero_out": r.n_zero_out, "n_snapped": r.n_snapped, "n_saturated": r.n_saturated,
+                    "n_underflow": r.n_underflow})
     return out
 
 
@@ -370,7 +377,9 @@ def _result_dict(r: LayerResultT) -> Dict:
             "mu": r.stats.mu, "sigma": r.stats.sigma, "tau": r.tau,
             "fmt": {"nbits": r.fmt.nbits, "exp_bits": r.fmt.exp_bits, "man_bits": r.fmt.man_bits,
                     "scale_exp": r.fmt.scale_exp},
-            "status": r.status, "max_abs": r.max_abs, "n_right_mode": r.n_right_mode}
+            "status": r.status, "max_abs": r.max_abs, "n_right_mode": r.n_right_mode,
+            "n_zero_out": r.n_zero_out, "n_snapped": r.n_snapped, "n_saturated": r.n_saturated,
+            "n_underflow": r.n_underflow}
 
 
 def make_host_layer(g: torch.Tensor, out: torch.Tensor, mode: int, **kw) -> LayerT:
@@ -380,7 +389,8 @@ def make_host_layer(g: torch.Tensor, out: torch.Tensor, mode: int, **kw) -> Laye
     lay = LayerT(g.data_ptr() or None, out.data_ptr() or None, g.numel(), dtype_code(g), mode,
                  float(kw.get("S", 0.0)), int(kw.get("nbits", 0)), int(kw.get("rounding", ROUND_NEAREST)),
                  int(kw.get("seed", 0)), 0, int(kw.get("scale_mode", SCALE_CENTRED)), 0.0, 0.0,
-                 (kw["right_mode"].data_ptr() or None) if kw.get("right_mode") is not None else None)
+                 (kw["right_mode"].data_ptr() or None) if kw.get("right_mode") is not None else None,
+                 1 if kw.get("counters") else 0, 0)
     return lay
 
 

@@ -75,6 +75,7 @@ static lgn_status check_layer(const lgn_layer_t &d) {
         const size_t out_bytes = d.n * (d.dt == LGN_BF16 ? 2u : 4u);
         if (m < b + out_bytes && b < m + d.n) return LGN_ERR_INVALID_ARG;   // the output would overwrite the mask
     }
+    if (d.reserved != 0) return LGN_ERR_INVALID_ARG;
     if (d.use_override && !(d.sigma_override >= 0.0 && std::isfinite(d.mu_override) && std::isfinite(d.sigma_override)))
         return LGN_ERR_INVALID_ARG;
     return LGN_OK;
@@ -152,13 +153,14 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
         s.use_override = d.use_override ? 1 : 0;
         s.scale_mode = d.scale_mode;
         s.mask = static_cast<const uint8_t *>(d.right_mode);
+        s.counters = d.counters ? 1 : 0;
     }
 
     // one kernel per (type, mode, width, rounding) shared by all layers; the general one otherwise.
     // Extended statistics: the specialised kernels' second instances; mixed groups go general.
     bool any_ext = false, same = true;
     for (int k = 0; k < L; ++k) {
-        any_ext = any_ext || needs_ext_stats(st[k]);
+        any_ext = any_ext || needs_ext_stats(st[k]) || st[k].counters;
         same = same && st[k].dt == st[0].dt && variant_of(st[k].mode, st[k].nbits, st[k].rounding) ==
                                                    variant_of(st[0].mode, st[0].nbits, st[0].rounding);
     }
@@ -167,6 +169,8 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
     else if (same && st[0].mode == LGN_MODE_PRUNE) fn = compress_table(st[0].dt)[kVariantPruneExt];
     else if (same && st[0].mode == LGN_MODE_QUANTIZE)
         fn = compress_table(st[0].dt)[kVariantQuantExt0 + variant_of(st[0].mode, st[0].nbits, st[0].rounding) - 2];
+    if (any_ext || !same)                        // these kernels count for every layer of the call
+        for (int k = 0; k < L; ++k) st[k].counters = 1;
     int grid = persistent_ctas(fn);
     if (grid < 1) return LGN_ERR_CUDA;
 

@@ -535,10 +535,39 @@ __device__ __forceinline__ uint32_t prune_pair_bf16(uint32_t w, uint32_t r, floa
     return kept2 & ~dead2;
 }
 
+// What an apply tile counts for its layer's result record when asked to (COUNT): pruning: a =
+// outputs that are not zero, b = inputs above alpha (a - b of the kept ones were snapped to
+// +-alpha); quantisation: a = codes that are not zero, b = codes of the largest magnitude.
+struct TileCounts { uint32_t a = 0, b = 0; };
+
+// Counts of one chunk of a pruning tile, taken from the input chunk and the finished output
+// chunk, so that the elementwise forms above stay as they are.  Elements past the end of the
+// tensor were read as zeros and written as zeros: they count in neither.
+template <int DT>
+__device__ __forceinline__ void count_pruned_chunk(const Chunk &in, const Chunk &o, float tau, TileCounts &tc) {
+    if (DT == LGN_F32) {
+        #pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            tc.a += (o.w[k] & 0x7FFFFFFFu) != 0u ? 1u : 0u;
+            tc.b += fabsf(u2f(in.w[k])) > tau ? 1u : 0u;
+        }
+    } else {
+        const uint32_t ones = 0x00010001u, neg_tau2 = (0u - (f2u(tau) >> 16)) & 0xFFFFu;
+        uint32_t a2 = 0u, b2 = 0u;                         // two 16-bit lane counters each: at most 8 per chunk
+        #pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            a2 += __vminu2(o.w[k] & 0x7FFF7FFFu, ones);
+            b2 += __vminu2(__viaddmax_s16x2(in.w[k] & 0x7FFF7FFFu, neg_tau2 * ones, 0u), ones);   // max(|x| - alpha, 0) as patterns
+        }
+        tc.a += (a2 & 0xFFFFu) + (a2 >> 16);
+        tc.b += (b2 & 0xFFFFu) + (b2 >> 16);
+    }
+}
+
 // tau == 0 never reaches the fast forms' arithmetic (the tile is copied instead).
-template <int DT, bool FULL, int TILE = kTileElems>
+template <int DT, bool FULL, int TILE = kTileElems, bool COUNT = false>
 __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t tile_base, uint64_t n,
-                                           float tau, uint64_t seed, const Weyl &wy) {
+                                           float tau, uint64_t seed, const Weyl &wy, TileCounts *tc = nullptr) {
     constexpr int C = ElemTraits<DT>::kChunk;
     constexpr int kLoads = TILE / (kThreads * C);
     constexpr int kGroup = 1;                             // one chunk per buffer: the apply bodies need the registers
@@ -578,6 +607,7 @@ __device__ __forceinline__ void prune_tile(const void *g, void *out, uint64_t ti
                 }
             }
             store_chunk<DT, FULL>(out, i, n, o);
+            if constexpr (COUNT) count_pruned_chunk<DT>(v[j], o, tau, *tc);
         }
     });
 }
@@ -744,9 +774,10 @@ __device__ __forceinline__ uint32_t quant_pair_bf16(uint32_t w, uint32_t r, cons
 // not a multiple of 32, the first bits of the next lane (one warp shuffle), so
 // every store is an aligned 32-bit word of the little-endian bit stream.
 // `total_words` = words in the whole stream.
-template <int DT, int NBITS, bool SR, bool FAST, bool FULL, int TILE = kTileElems>
+template <int DT, int NBITS, bool SR, bool FAST, bool FULL, int TILE = kTileElems, bool COUNT = false>
 __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint64_t tile_base, uint64_t n,
-                                           uint64_t total_words, const QuantParams &q, uint64_t seed, const Weyl &wy) {
+                                           uint64_t total_words, const QuantParams &q, uint64_t seed, const Weyl &wy,
+                                           TileCounts *tc = nullptr) {
     constexpr int C = ElemTraits<DT>::kChunk;
     constexpr int B = C * NBITS;                           // bits per lane per load step: 32..128
     constexpr int NW = (B + 31) / 32;                      // words that hold a lane's bits
@@ -776,6 +807,11 @@ __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint6
                     #pragma unroll
                     for (int pr = 0; pr < 4; ++pr) {       // word pr of the block <-> elements 2pr, 2pr+1
                         const uint32_t two = quant_pair_bf16<NBITS, SR>(v[j].w[b * 4 + pr], rw[pr], pq);
+                        if constexpr (COUNT) {
+                            const uint32_t m0 = two & (q.sign_bit - 1u), m1 = (two >> NBITS) & (q.sign_bit - 1u);
+                            tc->a += (m0 != 0u ? 1u : 0u) + (m1 != 0u ? 1u : 0u);
+                            tc->b += (m0 == q.top ? 1u : 0u) + (m1 == q.top ? 1u : 0u);
+                        }
                         const int pos = (b * 8 + 2 * pr) * NBITS;
                         cw[pos >> 5] |= two << (pos & 31);
                         if ((pos & 31) + 2 * NBITS > 32) cw[(pos >> 5) + 1] |= two >> (32 - (pos & 31));
@@ -785,6 +821,11 @@ __device__ __forceinline__ void quant_tile(const void *g, uint32_t *codes, uint6
                     for (int e = 0; e < 8; ++e) {
                         const int k = b * 8 + e;
                         const uint32_t code = quant_elem<SR, FAST>(elem_bits<DT>(v[j], k), SR ? rand_h(r, e) : 0u, q);
+                        if constexpr (COUNT) {
+                            const uint32_t m = code & (q.sign_bit - 1u);
+                            tc->a += m != 0u ? 1u : 0u;
+                            tc->b += m == q.top ? 1u : 0u;
+                        }
                         const int pos = k * NBITS;         // a constant once the loops are unrolled
                         cw[pos >> 5] |= code << (pos & 31);
                         if ((pos & 31) + NBITS > 32) cw[(pos >> 5) + 1] |= code >> (32 - (pos & 31));

@@ -54,7 +54,8 @@ struct alignas(16) LayerState {          // written by the set-up launch, then r
     uint32_t            partial0;        // first slot of this layer in the partial array
     int32_t             dt, mode, nbits, rounding, use_override, scale_mode;
     const uint8_t      *mask;            // right-mode mask of a bi-modal gradient, or null
-    uint64_t            pad;
+    int32_t             counters;        // the apply tiles add their counts to result_out
+    int32_t             pad;
 };
 static_assert(sizeof(LayerState) == 128, "LayerState layout");
 
@@ -240,47 +241,72 @@ __device__ __noinline__ void run_stats_tile_slow(const LayerState &L, uint32_t t
     }
 }
 
+// The general bodies always count (they are not the fast path); `tc` may be null.
 template <int DT, int TILE>
 __device__ __noinline__ void prune_tile_general(const void *g, void *out, uint64_t base, uint64_t n,
-                                                float tau, uint64_t seed, const Weyl &wy) {
-    prune_tile<DT, false, TILE>(g, out, base, n, tau, seed, wy);
+                                                float tau, uint64_t seed, const Weyl &wy, TileCounts *tc) {
+    TileCounts local;
+    prune_tile<DT, false, TILE, true>(g, out, base, n, tau, seed, wy, &local);
+    if (tc) { tc->a += local.a; tc->b += local.b; }
 }
 
-template <int DT, bool INLINE_HOT, int TILE>
+// COUNT: the inlined hot body counts too (the instances that serve groups which ask for counters).
+template <int DT, bool INLINE_HOT, int TILE, bool COUNT = false>
 __device__ __forceinline__ void run_prune_tile(const void *g, void *out, uint64_t n, uint32_t tile,
-                                               float tau, uint64_t seed, const Weyl &wy) {
+                                               float tau, uint64_t seed, const Weyl &wy, TileCounts *tc = nullptr) {
     const uint64_t base = (uint64_t)tile * TILE;
     const bool tiny = tau > 0.f && tau < kPruneFastMin;       // alpha*2^-16 inexact, or alpha*eps could round to zero
-    if (INLINE_HOT && base + TILE <= n && !tiny) prune_tile<DT, true, TILE>(g, out, base, n, tau, seed, wy);
-    else                                         prune_tile_general<DT, TILE>(g, out, base, n, tau, seed, wy);
+    if (INLINE_HOT && base + TILE <= n && !tiny) prune_tile<DT, true, TILE, COUNT>(g, out, base, n, tau, seed, wy, tc);
+    else                                         prune_tile_general<DT, TILE>(g, out, base, n, tau, seed, wy, tc);
 }
 
 template <int DT, int NBITS, bool SR, int TILE>
 __device__ __noinline__ void quant_tile_general(const void *g, uint32_t *codes, uint64_t base, uint64_t n,
                                                 uint64_t total_words, const QuantParams &q, uint64_t seed,
-                                                const Weyl &wy) {
-    quant_tile<DT, NBITS, SR, false, false, TILE>(g, codes, base, n, total_words, q, seed, wy);
+                                                const Weyl &wy, TileCounts *tc) {
+    TileCounts local;
+    quant_tile<DT, NBITS, SR, false, false, TILE, true>(g, codes, base, n, total_words, q, seed, wy, &local);
+    if (tc) { tc->a += local.a; tc->b += local.b; }
 }
 
-template <int DT, int NBITS, bool SR, bool INLINE_HOT, int TILE>
+template <int DT, int NBITS, bool SR, bool INLINE_HOT, int TILE, bool COUNT = false>
 __device__ __forceinline__ void run_quant_tile(const void *g, void *out, uint64_t n, uint32_t tile,
-                                               const QuantParams &q, uint64_t seed, const Weyl &wy) {
+                                               const QuantParams &q, uint64_t seed, const Weyl &wy, TileCounts *tc = nullptr) {
     const uint64_t base = (uint64_t)tile * TILE;
     const uint64_t total_words = (n * (uint64_t)NBITS + 31) >> 5;
     uint32_t *codes = static_cast<uint32_t *>(out);
     if (INLINE_HOT && base + TILE <= n && q.K >= 1 && q.K <= 255)
-        quant_tile<DT, NBITS, SR, true, true, TILE>(g, codes, base, n, total_words, q, seed, wy);
+        quant_tile<DT, NBITS, SR, true, true, TILE, COUNT>(g, codes, base, n, total_words, q, seed, wy, tc);
     else
-        quant_tile_general<DT, NBITS, SR, TILE>(g, codes, base, n, total_words, q, seed, wy);
+        quant_tile_general<DT, NBITS, SR, TILE>(g, codes, base, n, total_words, q, seed, wy, tc);
+}
+
+// Adds a tile's counts to its layer's result record: one warp-wide sum and, from lane 0, one
+// atomic per field.  finalize_layer has stored the record, with the counters at their starting
+// values (see there), before any apply tile of the layer can run.
+__device__ __forceinline__ void flush_counts(const LayerState &L, const TileCounts &tc) {
+    if (!L.counters || L.result_out == nullptr) return;
+    const unsigned long long a = __reduce_add_sync(0xFFFFFFFFu, tc.a), b = __reduce_add_sync(0xFFFFFFFFu, tc.b);
+    if ((threadIdx.x & 31) != 0) return;
+    lgn_layer_result_t *r = L.result_out;
+    if (L.mode == LGN_MODE_PRUNE) {
+        atomicAdd(reinterpret_cast<unsigned long long *>(&r->n_zero_out), 0ull - a);    // starts at n
+        atomicAdd(reinterpret_cast<unsigned long long *>(&r->n_snapped), a - b);        // kept but not above alpha
+    } else {
+        atomicAdd(reinterpret_cast<unsigned long long *>(&r->n_zero_out), 0ull - a);    // starts at n
+        atomicAdd(reinterpret_cast<unsigned long long *>(&r->n_underflow), 0ull - a);   // starts at nnz
+        atomicAdd(reinterpret_cast<unsigned long long *>(&r->n_saturated), b);
+    }
 }
 
 // run-time dispatch for groups whose layers differ in type, mode or width
 template <int DT>
 __device__ __forceinline__ void run_quant_tile_any(const void *g, void *out, uint64_t n, uint32_t tile, int nbits,
-                                                   const QuantParams &q, bool sr, uint64_t seed, const Weyl &wy) {
+                                                   const QuantParams &q, bool sr, uint64_t seed, const Weyl &wy,
+                                                   TileCounts *tc) {
     #define LGN_Q(NB) \
-        if (sr) run_quant_tile<DT, NB, true, false, kTileElems>(g, out, n, tile, q, seed, wy); \
-        else    run_quant_tile<DT, NB, false, false, kTileElems>(g, out, n, tile, q, seed, wy);
+        if (sr) run_quant_tile<DT, NB, true, false, kTileElems>(g, out, n, tile, q, seed, wy, tc); \
+        else    run_quant_tile<DT, NB, false, false, kTileElems>(g, out, n, tile, q, seed, wy, tc);
     switch (nbits) {
         case 4: LGN_Q(4) break;
         case 5: LGN_Q(5) break;
@@ -360,6 +386,12 @@ static __device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn
         lgn_layer_result_t r;
         r.stats = st; r.tau = tau_used; r.fmt = fmt; r.status = LGN_OK;
         r.max_abs = acc.amax; r.n_right_mode = L.mask ? acc.right : 0ull;
+        // Counters start where the apply tiles' atomics (flush_counts) leave the final values:
+        // zeros out = n - nonzero outputs; underflows = nnz - nonzero codes (a nonzero code
+        // always comes from a nonzero input).
+        r.n_zero_out = L.counters ? st.n : 0ull;
+        r.n_underflow = (L.counters && L.mode == LGN_MODE_QUANTIZE) ? st.nnz : 0ull;
+        r.n_snapped = 0ull; r.n_saturated = 0ull;
         *L.result_out = r;
     }
     __threadfence();
@@ -496,23 +528,27 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
                 if (!sm_flag) continue;                            // timed out: skip the tile, keep draining
                 ready_layer = (int)sg.layer;
             }
+            // The instances with extended statistics also take the counters of the result record
+            // (EXT is "everything beyond the plain path"); so does the general kernel.
+            TileCounts tc;
             if constexpr (kSpecial && MODE == LGN_MODE_PRUNE) {
-                run_prune_tile<DT, true, TILE>(L.g, L.out, L.n, tile, __ldcg(&D->tau), L.seed, wy);
+                run_prune_tile<DT, true, TILE, EXT>(L.g, L.out, L.n, tile, __ldcg(&D->tau), L.seed, wy, EXT ? &tc : nullptr);
             } else if constexpr (kSpecial && MODE == LGN_MODE_QUANTIZE) {
                 const QuantParams q = load_quant_params(D);
-                run_quant_tile<DT, NBITS, SR != 0, true, TILE>(L.g, L.out, L.n, tile, q, L.seed, wy);
+                run_quant_tile<DT, NBITS, SR != 0, true, TILE, EXT>(L.g, L.out, L.n, tile, q, L.seed, wy, EXT ? &tc : nullptr);
             } else if constexpr (!kSpecial) {
                 if (L.mode == LGN_MODE_PRUNE) {
                     const float tau = __ldcg(&D->tau);
-                    if (L.dt == LGN_BF16) run_prune_tile<LGN_BF16, false, kTileElems>(L.g, L.out, L.n, tile, tau, L.seed, wy);
-                    else                  run_prune_tile<LGN_F32, false, kTileElems>(L.g, L.out, L.n, tile, tau, L.seed, wy);
+                    if (L.dt == LGN_BF16) run_prune_tile<LGN_BF16, false, kTileElems>(L.g, L.out, L.n, tile, tau, L.seed, wy, &tc);
+                    else                  run_prune_tile<LGN_F32, false, kTileElems>(L.g, L.out, L.n, tile, tau, L.seed, wy, &tc);
                 } else {
                     const QuantParams q = load_quant_params(D);
                     const bool sr = L.rounding == LGN_ROUND_STOCHASTIC;
-                    if (L.dt == LGN_BF16) run_quant_tile_any<LGN_BF16>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed, wy);
-                    else                  run_quant_tile_any<LGN_F32>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed, wy);
+                    if (L.dt == LGN_BF16) run_quant_tile_any<LGN_BF16>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed, wy, &tc);
+                    else                  run_quant_tile_any<LGN_F32>(L.g, L.out, L.n, tile, L.nbits, q, sr, L.seed, wy, &tc);
                 }
             }
+            if constexpr (EXT || !kSpecial) flush_counts(L, tc);
         }
     }
 }

@@ -29,8 +29,8 @@ def test_every_declared_symbol_is_exported(lgn):
 def test_struct_sizes_match_header(lgn):
     assert C.sizeof(lgn.StatsT) == 48
     assert C.sizeof(lgn.FpFormatT) == 16
-    assert C.sizeof(lgn.LayerT) == 88
-    assert C.sizeof(lgn.LayerResultT) == 88
+    assert C.sizeof(lgn.LayerT) == 96
+    assert C.sizeof(lgn.LayerResultT) == 120
 
 
 def test_status_strings(lgn):
@@ -138,7 +138,8 @@ def test_device_entry_points_reject_bad_arguments_before_any_cuda_call(lgn):
     # grouped
     def layer(**kw):
         d = dict(g=A, out=B, n=100, dt=0, mode=0, S=0.8, nbits=6, rounding=0, seed=0,
-                 use_override=0, scale_mode=0, mu_override=0.0, sigma_override=0.0, right_mode=None)
+                 use_override=0, scale_mode=0, mu_override=0.0, sigma_override=0.0, right_mode=None,
+                 counters=0, reserved=0)
         d.update(kw)
         return lgn.LayerT(*[d[f[0]] for f in lgn.LayerT._fields_])
     def call(l, ws_bytes=None, res=0x300000, n=1):
@@ -159,6 +160,7 @@ def test_device_entry_points_reject_bad_arguments_before_any_cuda_call(lgn):
     assert call(layer(mode=1, right_mode=0x400000)) == INVALID        # a mask belongs to pruning
     assert call(layer(scale_mode=1)) == INVALID                       # a scale mode belongs to quantisation
     assert call(layer(mode=1, scale_mode=2)) == INVALID
+    assert call(layer(reserved=3)) == INVALID                         # must be zero
     assert call(layer(), ws_bytes=16) == WORKSPACE
     assert call(layer(), res=None) == INVALID
     assert call(layer(), n=-1) == INVALID
