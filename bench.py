@@ -363,15 +363,22 @@ class Prepared:
         return total, per
 
 
-# What the counters of one ncu capture say bounds each kind of workload (profiles/): fp32 pruning
-# moves the algorithmic bytes at the HBM rate; the other bodies execute 22-34 instructions per
-# element and sit between the HBM roof and the issue-slot ceiling.
-def roofline_of(name, alg_bytes, per_step_ms):
+# Roofs of one workload.  HBM: the measured copy rate.  The two instruction roofs come from one ncu
+# capture per kind of workload (profiles/issue_ceilings.json: instructions and integer-ALU
+# instructions per element): every issue slot used (148 SMs x 4 schedulers x 32 lanes per clock),
+# or every lane of the integer ALU pipe used (148 x 64 per clock), at the SM clock sampled during
+# the run.  `bound` names the lowest roof: "hbm", or "alu" where the ALU pipe's lies below it
+# (bf16 FP6), and `frac` is measured against that roof; `frac_hbm` is always against the copy rate.
+SMS, ISSUE_LANES, ALU_LANES = 148, 128, 64
+
+
+def roofline_of(name, alg_bytes, per_step_ms, sm_mhz=None):
     peak, peak_kind = read_peak()
     kern_ms = statistics.mean(per_step_ms)
     achieved = alg_bytes / (kern_ms * 1e-3) / 1e9
     r = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-         "traffic": None, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
+         "traffic": None, "peak_kind": f"of {peak_kind}", "frac_hbm": achieved / peak,
+         "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
          "kernel": "compress_kernel", "algorithmic_bytes_per_launch": alg_bytes,
          "best_ms": min(per_step_ms), "median_ms": statistics.median(per_step_ms)}
     try:
@@ -382,10 +389,20 @@ def roofline_of(name, alg_bytes, per_step_ms):
     except Exception:
         pass
     try:
+        w = WORKLOADS[name]
+        fam = f"{w['dtype']}_{'prune' if w['mode'] == 'prune' else 'quant' + str(w.get('nbits', 6))}"
         with open(os.path.join(ROOT, "profiles", "issue_ceilings.json")) as f:
-            ic = json.load(f).get(name)
-        if ic:
-            r["issue_ceiling"] = ic        # instructions per element (ncu) and the GB/s at which every issue slot is used
+            ic = json.load(f)
+        c = ic.get(fam)
+        if c and ic.get("library_sha") == lib_sha():
+            bpe = bytes_per_elem(2 if w["dtype"] == "bf16" else 4, w["mode"], w.get("nbits", 6))
+            hz = (sm_mhz or 1965.0) * 1e6
+            issue = SMS * ISSUE_LANES * hz / c["instr_per_elem"] * bpe / 1e9
+            alu = SMS * ALU_LANES * hz / c["alu_per_elem"] * bpe / 1e9
+            r["instruction_roofs"] = {"issue_GBps": issue, "alu_GBps": alu, "instr_per_elem": c["instr_per_elem"],
+                                      "alu_instr_per_elem": c["alu_per_elem"], "sm_mhz": hz / 1e6}
+            if alu < peak:
+                r.update(bound="alu", peak=alu, frac=achieved / alu, peak_kind="ALU-pipe lanes x SM clock / ALU instructions per element")
     except Exception:
         pass
     return r
@@ -474,7 +491,7 @@ def run_ours(args):
                    "parallelism": f"replicas x{world}"},
         "elements_per_s": world * P.total_elems / (ms_per_step * 1e-3),
         "gpu_launches": args.steps * lgn.lgn_launches_per_call(len(tensors)),
-        "roofline": roofline_of(args.workload, P.alg_bytes, per_step_ms),
+        "roofline": roofline_of(args.workload, P.alg_bytes, per_step_ms, clocks.get("sm_mhz") if clocks else None),
         "clocks": clocks,
         "wall_s": wall,
     }
