@@ -329,8 +329,30 @@ __host__ __device__ inline int floor_log2_f32(float a) {
     return top - 149;
 }
 
+// choose_format with the candidate splits spread over the lanes of a warp (lane k evaluates Eq. 4
+// for n2 = k + 1): the same arithmetic per candidate and the same choice (the smallest n2 among
+// the minima) as the sequential form, in the time of one evaluation instead of nbits - 1.
+// All 32 lanes call.
+__device__ __forceinline__ void choose_format_warp(double mu, double sigma, int nbits, lgn_fp_format_t &f) {
+    const double s = clamp_sigma(sigma);
+    int n2 = (int)(threadIdx.x & 31) + 1;
+    double eta = n2 <= nbits - 1 ? expected_rel_err(s, nbits - 1 - n2, n2) : __longlong_as_double(0x7FF0000000000000ll);
+    #pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const double oe = __shfl_down_sync(0xFFFFFFFFu, eta, off);
+        const int on = __shfl_down_sync(0xFFFFFFFFu, n2, off);
+        if (oe < eta || (oe == eta && on < n2)) { eta = oe; n2 = on; }
+    }
+    n2 = __shfl_sync(0xFFFFFFFFu, n2, 0);
+    f.nbits = nbits;
+    f.exp_bits = n2;
+    f.man_bits = nbits - 1 - n2;
+    f.scale_exp = (int32_t)floor(mu / kLn2 + 0.5);
+}
+
 // Adds up a layer's partials (thread t takes slots t, t+kThreads, ... in order,
-// then the fixed tree), turns them into mu, sigma, and evaluates the closed form.
+// then the fixed tree), turns them into mu, sigma, and evaluates the closed form (on warp 0:
+// every lane carries the same values, lane 0 stores them).
 static __device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn *D, const Partial *partials, double *sm) {
     StatsAcc acc;
     for (uint32_t t = threadIdx.x; t < L.ntiles; t += kThreads) {
@@ -342,7 +364,13 @@ static __device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn
         acc.amax = fmaxf(acc.amax, __ldcg(&p->amax));
     }
     block_reduce(acc, sm);
-    if (threadIdx.x != 0) return;
+    if (threadIdx.x >= 32) return;
+    acc.s1 = __shfl_sync(0xFFFFFFFFu, acc.s1, 0);
+    acc.s2 = __shfl_sync(0xFFFFFFFFu, acc.s2, 0);
+    acc.cnt = __shfl_sync(0xFFFFFFFFu, acc.cnt, 0);
+    acc.right = __shfl_sync(0xFFFFFFFFu, acc.right, 0);
+    acc.amax = __shfl_sync(0xFFFFFFFFu, acc.amax, 0);
+    const bool lead = threadIdx.x == 0;
 
     lgn_stats_t st;
     st.n = L.n;
@@ -358,7 +386,7 @@ static __device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn
         st.sum_ln = acc.s1 * kLn2;
         st.sum_ln2 = acc.s2 * kLn2 * kLn2;
     }
-    if (L.stats_out) *L.stats_out = st;
+    if (lead && L.stats_out) *L.stats_out = st;
 
     const double mu = L.use_override ? L.mu_override : st.mu;
     const double sigma = L.use_override ? L.sigma_override : st.sigma;
@@ -370,18 +398,19 @@ static __device__ __noinline__ void finalize_layer(const LayerState &L, LayerDyn
         const double zero_frac = 1.0 - (double)(L.mask ? acc.right : st.nnz) / (double)st.n;
         const double tau = acc.cnt ? threshold_for(mu, sigma, zero_frac, L.S) : 0.0;
         const float t = (L.dt == LGN_BF16) ? snap_threshold_bf16(tau) : snap_threshold_f32(tau);
-        D->tau = t;
+        if (lead) D->tau = t;
         tau_used = (double)t;
     } else if (L.mode == LGN_MODE_QUANTIZE) {
         if (acc.cnt) {
-            choose_format(mu, sigma, L.nbits, fmt);
+            choose_format_warp(mu, sigma, L.nbits, fmt);
             if (L.scale_mode == LGN_SCALE_FROM_MAX)               // Algorithm 1: the maximum in the top binade
                 fmt.scale_exp = floor_log2_f32(acc.amax) - ((1 << (fmt.exp_bits - 1)) - 1);
         } else {                                              // all zero: every code is 0 anyway
             fmt.nbits = L.nbits; fmt.exp_bits = 1; fmt.man_bits = L.nbits - 2; fmt.scale_exp = 0;
         }
-        D->q = make_quant_params(fmt);
+        if (lead) D->q = make_quant_params(fmt);
     }
+    if (!lead) return;
     if (L.result_out) {
         lgn_layer_result_t r;
         r.stats = st; r.tau = tau_used; r.fmt = fmt; r.status = LGN_OK;
