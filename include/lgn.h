@@ -263,10 +263,10 @@ typedef struct {
     /* Nonzero: the apply pass also counts what it did to this layer (n_zero_out .. n_underflow
      * of the result record).  The counts cost the integer pipe a few instructions per element
      * (measured on B200: a call takes 10 % (fp32 FP6) to 30 % (bf16 pruning) longer), so they
-     * are taken only by a second set of kernels, the one
-     * that also serves right_mode and LGN_SCALE_FROM_MAX: a call runs through it, and every
-     * layer of the call then gets its counts, as soon as one layer asks for any of the three,
-     * and so does every call whose layers differ in type, mode, width or rounding. */
+     * are taken only when asked for: as soon as one layer of a call sets this field, every
+     * layer of that call gets its counts (the call then runs through the second set of kernel
+     * instances, the one that also serves right_mode and LGN_SCALE_FROM_MAX); a call whose
+     * layers differ in type, mode, width or rounding always counts. */
     int32_t      counters;
     int32_t      reserved;   /* 0 */
 } lgn_layer_t;

@@ -561,10 +561,13 @@ compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Se
             // (EXT is "everything beyond the plain path"); so does the general kernel.
             TileCounts tc;
             if constexpr (kSpecial && MODE == LGN_MODE_PRUNE) {
-                run_prune_tile<DT, true, TILE, EXT>(L.g, L.out, L.n, tile, __ldcg(&D->tau), L.seed, wy, EXT ? &tc : nullptr);
+                const float tau = __ldcg(&D->tau);
+                if (EXT && L.counters) run_prune_tile<DT, true, TILE, EXT>(L.g, L.out, L.n, tile, tau, L.seed, wy, &tc);
+                else                   run_prune_tile<DT, true, TILE, false>(L.g, L.out, L.n, tile, tau, L.seed, wy, nullptr);
             } else if constexpr (kSpecial && MODE == LGN_MODE_QUANTIZE) {
                 const QuantParams q = load_quant_params(D);
-                run_quant_tile<DT, NBITS, SR != 0, true, TILE, EXT>(L.g, L.out, L.n, tile, q, L.seed, wy, EXT ? &tc : nullptr);
+                if (EXT && L.counters) run_quant_tile<DT, NBITS, SR != 0, true, TILE, EXT>(L.g, L.out, L.n, tile, q, L.seed, wy, &tc);
+                else                   run_quant_tile<DT, NBITS, SR != 0, true, TILE, false>(L.g, L.out, L.n, tile, q, L.seed, wy, nullptr);
             } else if constexpr (!kSpecial) {
                 if (L.mode == LGN_MODE_PRUNE) {
                     const float tau = __ldcg(&D->tau);
