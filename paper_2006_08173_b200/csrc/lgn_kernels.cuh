@@ -452,8 +452,15 @@ constexpr int kAny = -1;                      // template value: decided per lay
 // layers may ask for the extended statistics tile (a right-mode mask, max|g|);
 // every specialised kernel exists without and (as a second instance) with it, so a
 // group that does not ask pays nothing for it.
+// Resident CTAs per SM the grouped kernel is compiled for: three (80 registers, no spills), which
+// measured 2-4 % faster than four (64 registers, some spills) on every fp32 workload and on bf16
+// with 32768-element tiles; the bf16 instances with 65536-element tiles keep four (ResNet-50 bf16
+// pruning: -1.6 % at three); two is slower everywhere.
+template <int DT, int TILE>
+constexpr int compress_min_ctas() { return (DT == LGN_BF16 && TILE > kTileElems) ? kMinCtas : kMinCtas - 1; }
+
 template <int DT, int MODE, int NBITS, int SR, bool EXT = false, int TILE = kTileElems>
-__global__ void __launch_bounds__(kThreads, kMinCtas)
+__global__ void __launch_bounds__(kThreads, compress_min_ctas<DT, TILE>())
 compress_kernel(WsHeader *hdr, const LayerState *states, LayerDyn *dyn, const Segment *segs,
                 int num_layers, uint32_t total_items, Partial *partials) {
     __shared__ double sm_red[5 * kWarps];
