@@ -557,9 +557,9 @@ def run_aux(args):
         out = torch.empty(16, dtype=torch.uint8, device=dev)
         raw, gp, code, st_ = lgn.raw(), g.data_ptr(), lgn.dtype_code(g), torch.cuda.current_stream().cuda_stream
         call = lambda: raw.lgn_quantile(gp, n, code, 0.997, out.data_ptr(), ws.data_ptr(), ws.numel(), st_)
-        alg_bytes = float(n * esize)                    # one read of the tensor (the fp32 selection reads it twice)
-        kernel = "quantile_top_kernel (+ quantile_low_kernel for fp32)"
-        launches = 5 if esize == 4 else 3
+        alg_bytes = float(n * esize)                    # one read of the tensor
+        kernel = "quantile_count_kernel (behind quantile_sample_kernel; the histogram kernels return at once)"
+        launches = (4 if esize == 4 else 3) if n >= 2 ** 24 else (2 if esize == 4 else 1)
     elif w["kind"] in ("bimodal", "maxscale"):
         # one layer of the grouped call with the variant switched on
         if w["kind"] == "bimodal":

@@ -31,6 +31,44 @@ def test_quantile_parity(lgn, oracle, dtype, n):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
+def test_quantile_parity_bracket_path(lgn, oracle, dtype):
+    """From 2^24 elements the selection reads the tensor once, around a bracket taken from a sample."""
+    g = synth.lognormal_tensor(2 ** 24 + 5, -12.0, 2.0, 0.4, seed=17, dtype=dtype, device="cuda")
+    for q in (0.0, 0.003, 0.5, 0.9, 0.997, 0.99999, 1.0):
+        check(lgn, oracle, g, q)
+    g = synth.lognormal_tensor(2 ** 26 + 8 * 3 + 1, -9.0, 3.0, 0.7, seed=18, dtype=dtype, device="cuda")
+    check(lgn, oracle, g, 0.997)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_quantile_when_the_bracket_fails(lgn, oracle, dtype):
+    """Inputs on which the one-read selection has to give up (more elements inside the bracket than its
+    list holds; a sample without a nonzero element) and the two-pass selection answers instead."""
+    n = 2 ** 24 + 11
+    gen = torch.Generator(device="cuda").manual_seed(3)
+    # all values equal; all values in one bin of the upper 15 bits; every value distinct in a narrow band
+    const = torch.full((n,), -3.0, device="cuda").to(dtype)
+    const[::3] = 0
+    band = (1.0 + torch.rand(n, device="cuda", generator=gen) / 128.0).to(dtype)
+    for g in (const, band):
+        for q in (0.5, 0.997):
+            check(lgn, oracle, g, q)
+    # a handful of nonzero elements that the sample is unlikely to meet
+    sparse = torch.zeros(n, dtype=dtype, device="cuda")
+    sparse[torch.tensor([5, 77_777, 1_000_003, 14_999_999, n - 1], device="cuda")] = torch.tensor([0.5, -2.0, 1e-3, 8.0, -0.25], device="cuda").to(dtype)
+    for q in (0.0, 0.5, 1.0):
+        check(lgn, oracle, sparse, q)
+    # magnitudes in increasing order (the sample still represents them), and in two populations far apart
+    ramp = synth.lognormal_tensor(n, -12.0, 2.0, 0.2, seed=4, dtype=dtype, device="cuda")
+    ramp = ramp[torch.argsort(ramp.float().abs())].contiguous()
+    check(lgn, oracle, ramp, 0.997)
+    two = torch.cat([synth.lognormal_tensor(n // 2, -20.0, 1.0, 0.1, seed=5, dtype=dtype, device="cuda"),
+                     synth.lognormal_tensor(n - n // 2, 2.0, 0.5, 0.0, seed=6, dtype=dtype, device="cuda")])
+    for q in (0.4, 0.5, 0.6):
+        check(lgn, oracle, two, q)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
 def test_quantile_special_inputs(lgn, oracle, dtype):
     z = torch.zeros(70_000, dtype=dtype, device="cuda")
     assert lgn.lgn_quantile(z, 0.997) == {"value": 0.0, "nnz": 0}
