@@ -182,17 +182,25 @@ lgn_status lgn_allocate_sparsity(const lgn_alloc_layer_t *layers, int num_layers
                                  double S, double s_max, double *S_out, double *achieved);
 
 /* lgn_quantile: the order statistic of rank ceil(q * nnz) (1-based) of |g| over the
- * nonzero elements, exactly, by a radix selection on the magnitude patterns (one pass
- * over a bf16 tensor, two over an fp32 tensor).  With the layer's mu and sigma,
- * k = (ln(value) - mu) / sigma is the cut used above.
+ * nonzero elements, exactly, by selection on the magnitude patterns.  With the layer's
+ * mu and sigma, k = (ln(value) - mu) / sigma is the cut used above.
  *   g        device, n elements of dt, 32-byte aligned
  *   q        in [0, 1]
  *   out_dev  device, 16 bytes, 16-byte aligned: { float value; uint32_t pad; uint64_t nnz }
  *            (value 0 when the tensor has no nonzero element)
- *   ws       device scratch of lgn_quantile_workspace_bytes() bytes, 16-byte aligned
+ *   ws       device scratch of lgn_quantile_workspace_bytes() bytes (4.5 MiB), 16-byte aligned
+ * Tensors below 2^24 elements: radix selection, one read of a bf16 tensor, two of an fp32
+ * tensor.  Larger tensors are read once (plus a sample of at least 2^21 elements): a
+ * bracket around the wanted element is taken from the sample, the full read counts what
+ * lies below it and sets aside what lies inside, and the answer is picked among those; if
+ * the bracket turns out not to hold the element, or holds more than the scratch has room
+ * for (2^16 fp32 patterns per sixteenth of the bracket; 4096 bf16 values), the radix
+ * selection runs after all.  For fp32 and q far from 0 and 1 the sample needed grows with
+ * n^2 q (1 - q); where it would pass n / 8 the radix selection is used at once.  The result
+ * is exact in every case.
  * n must be below 2^32 (the histogram bins are 32-bit counters): a larger n returns
  * LGN_ERR_UNSUPPORTED and nothing is enqueued.
- * Three (bf16) or five (fp32) small launches on `stream`, no allocation. */
+ * One memset and one to four launches on `stream`, no allocation. */
 typedef struct { float value; uint32_t pad; uint64_t nnz; } lgn_quantile_t;
 size_t     lgn_quantile_workspace_bytes(void);
 lgn_status lgn_quantile(const void *g, uint64_t n, lgn_dtype dt, double q, lgn_quantile_t *out_dev,

@@ -56,7 +56,7 @@ constexpr uint32_t kQListCap = 1u << 20;            // fp32 patterns the count p
 constexpr int kQBuckets = 16;                       // in this many lists by the leading bits of (pattern - lo)
 constexpr uint32_t kQBucketCap = kQListCap / kQBuckets;
 constexpr int kQCountThreads = 512;
-constexpr int kQRoundSteps = 4;                     // a round of the count pass: this many steps of kQInFlight chunks per thread (256 KiB)
+constexpr int kQRoundSteps = 2;                     // a round of the count pass: this many steps of kQInFlight chunks per thread (128 KiB)
 constexpr int kQCoarse = 128;                       // groups of 256 bins whose sums the sample pass also keeps
 constexpr int kQSideBins = 4096;                    // fp32: patterns staged per CTA; bf16: values a bracket may span;
                                                     // also the bins of one radix pass over the list
@@ -165,21 +165,26 @@ __device__ __forceinline__ unsigned long long own_sum(const uint32_t *hist) {
     return s;
 }
 
-// Finds the bin that holds rank `rank` (1-based, 1 <= rank <= total): the thread whose PER
-// bins contain it announces itself, then warp 0 scans those bins 32 at a time.  The answer
-// comes back in every thread (through shared memory).  All threads must call.
+// Finds the bins that hold the ranks rank[0] and rank[1] (1-based, 1 <= rank <= total; 0: none
+// wanted): the thread whose PER bins contain a rank announces itself, then warp w scans the bins
+// of rank[w]'s owner, 32 at a time.  The answers come back in every thread (through shared
+// memory).  All threads must call.
 template <int PER, bool SHARED>
-__device__ __forceinline__ void locate(const uint32_t *hist, unsigned long long rank, unsigned long long mine,
-                                       unsigned long long before, uint32_t *bin, unsigned long long *rank_in_bin) {
-    __shared__ uint32_t sm_owner, sm_bin;
-    __shared__ unsigned long long sm_before, sm_rib;
-    __syncthreads();                                       // the previous call's answer has been read
-    if (rank > before && rank <= before + mine) { sm_owner = threadIdx.x; sm_before = before; }
+__device__ __forceinline__ void locate_pair(const uint32_t *hist, const unsigned long long (&rank)[2], unsigned long long mine,
+                                            unsigned long long before, uint32_t (&bin)[2], unsigned long long (&rank_in_bin)[2]) {
+    __shared__ uint32_t sm_owner[2], sm_bin[2];
+    __shared__ unsigned long long sm_before[2], sm_rib[2];
+    __syncthreads();                                       // the previous call's answers have been read
+    #pragma unroll
+    for (int w = 0; w < 2; ++w)
+        if (rank[w] > before && rank[w] <= before + mine) { sm_owner[w] = threadIdx.x; sm_before[w] = before; }
     __syncthreads();
-    if (threadIdx.x < 32) {
-        const int lane = threadIdx.x;
-        const uint32_t base = sm_owner * PER;
-        unsigned long long cum = sm_before;
+    const int w = threadIdx.x >> 5;
+    const unsigned long long want = w == 0 ? rank[0] : rank[1];
+    if (w < 2 && want != 0ull) {
+        const int lane = threadIdx.x & 31;
+        const uint32_t base = sm_owner[w] * PER;
+        unsigned long long cum = sm_before[w];
         constexpr int STEPS = (PER + 31) / 32;
         uint32_t counts[STEPS];
         #pragma unroll
@@ -187,22 +192,32 @@ __device__ __forceinline__ void locate(const uint32_t *hist, unsigned long long 
             counts[s] = s * 32 + lane < PER ? (SHARED ? hist[base + s * 32 + lane] : __ldcg(hist + base + s * 32 + lane)) : 0u;
         #pragma unroll
         for (int s = 0; s < STEPS; ++s) {
-            const int j = s * 32;
             const uint32_t c = counts[s];
             unsigned long long incl = c;
             #pragma unroll
             for (int d = 1; d < 32; d <<= 1) { const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, incl, d); if (lane >= d) incl += t; }
-            const bool hit = c != 0u && rank > cum + incl - c && rank <= cum + incl;
+            const bool hit = c != 0u && want > cum + incl - c && want <= cum + incl;
             if (__any_sync(0xFFFFFFFFu, hit)) {
-                if (hit) { sm_bin = base + j + lane; sm_rib = rank - (cum + incl - c); }
+                if (hit) { sm_bin[w] = base + s * 32 + lane; sm_rib[w] = want - (cum + incl - c); }
                 break;
             }
             cum += __shfl_sync(0xFFFFFFFFu, incl, 31);
         }
     }
     __syncthreads();
-    *bin = sm_bin;
-    *rank_in_bin = sm_rib;
+    #pragma unroll
+    for (int k = 0; k < 2; ++k) { bin[k] = sm_bin[k]; rank_in_bin[k] = sm_rib[k]; }
+}
+
+template <int PER, bool SHARED>
+__device__ __forceinline__ void locate(const uint32_t *hist, unsigned long long rank, unsigned long long mine,
+                                       unsigned long long before, uint32_t *bin, unsigned long long *rank_in_bin) {
+    const unsigned long long ranks[2] = { rank, 0ull };
+    uint32_t bins[2];
+    unsigned long long ribs[2];
+    locate_pair<PER, SHARED>(hist, ranks, mine, before, bins, ribs);
+    *bin = bins[0];
+    *rank_in_bin = ribs[0];
 }
 
 // ---------------------------------------------------------------- histogram path
@@ -331,24 +346,19 @@ quantile_sample_kernel(const void *g, uint64_t n, uint32_t nsample, uint32_t ste
     if (m > 0) {                                           // uniform over the CTA
         const double centre = q * (double)m, dev = kQSigmas * sqrt((double)m * q * (1.0 - q)) + 2.0;
         const double r_lo = floor(centre - dev), r_hi = ceil(centre + dev);
-        uint32_t bin;
-        unsigned long long rib;
-        if (r_lo >= 1.0) {
-            locate<PER, false>(hist_sample, (unsigned long long)r_lo, mine, before, &bin, &rib);
-            lo = bin << 16;
-            if (lo < 1u) lo = 1u;
-        }
-        if (r_hi <= (double)m) {
-            locate<PER, false>(hist_sample, (unsigned long long)r_hi, mine, before, &bin, &rib);
-            hi = (bin + 1u) << 16;
-        }
+        const unsigned long long ranks[2] = { r_lo >= 1.0 ? (unsigned long long)r_lo : 0ull, r_hi <= (double)m ? (unsigned long long)r_hi : 0ull };
+        uint32_t bins[2];
+        unsigned long long ribs[2];
+        locate_pair<PER, false>(hist_sample, ranks, mine, before, bins, ribs);
+        if (ranks[0]) { lo = bins[0] << 16; if (lo < 1u) lo = 1u; }
+        if (ranks[1]) hi = (bins[1] + 1u) << 16;
     }
     if (threadIdx.x == 0) { ctl->lo = lo; ctl->width = hi - lo; }
 }
 
 // The full read.  Registers count the nonzero elements and those at or above lo; an
 // element inside the bracket (rare) is set aside.  The tensor is handed out in rounds of
-// 256 KiB through a counter, one round ahead (CTAs do not get equal shares of the memory
+// 128 KiB through a counter, one round ahead (CTAs do not get equal shares of the memory
 // system: with equal static shares the slowest finished 25 to 45 % after the first).  The
 // last CTA finishes.
 template <int DT>
