@@ -15,6 +15,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <type_traits>
 
 #include <cuda_runtime.h>
 
@@ -178,19 +179,23 @@ prefix_encode_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host
         // short codes of the eight elements, first stream bit in bit 0
         uint32_t sb = 0u, q = 0u, vm = 0u;
         unsigned long long cuts = 0ull;                          // 5 bits per element: q after the element
-        #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const uint32_t pat = p[k];
-            const bool in = (uint32_t)k < nvalid;
-            const bool nz = in && pat != 0u;
-            const bool al = in && (pat & ~kSign) == tpc;
-            const uint32_t code = al ? ((pat & kSign) ? 5u : 1u) : (nz ? 3u : 0u);
-            sb |= code << q;
-            q += (in ? 1u : 0u) + (nz ? 1u : 0u) + (al ? 1u : 0u);
-            if (nz && !al) vm |= 1u << k;
-            cuts |= (unsigned long long)q << (5 * k);
-            pay[k][threadIdx.x] = pat;
-        }
+        auto classify = [&](auto whole) {                        // whole: all eight elements exist (every block but the last)
+            #pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t pat = p[k];
+                const bool in = decltype(whole)::value || (uint32_t)k < nvalid;
+                const bool nz = in && pat != 0u;
+                const bool al = in && (pat & ~kSign) == tpc;
+                const uint32_t code = al ? ((pat & kSign) ? 5u : 1u) : (nz ? 3u : 0u);
+                sb |= code << q;
+                q += (in ? 1u : 0u) + (nz ? 1u : 0u) + (al ? 1u : 0u);
+                if (nz && !al) vm |= 1u << k;
+                cuts |= (unsigned long long)q << (5 * k);
+                pay[k][threadIdx.x] = pat;
+            }
+        };
+        if ((b + 1) * LGN_PREFIX_BLOCK <= n) classify(std::true_type{});
+        else classify(std::false_type{});
         const uint32_t bits = q + W * __popc(vm);
 
         // exclusive scan of `bits` over the CTA
