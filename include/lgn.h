@@ -31,6 +31,11 @@
  *    enqueued.  A CUDA error at enqueue time is returned as LGN_ERR_CUDA.
  *  - Same inputs, seed and arguments give bitwise the same outputs and the same
  *    statistics on every run.
+ *  - With the environment variable LGN_LOG set (to anything but "" or "0"; read once
+ *    per process) the host side prints its decisions to stderr, one line each,
+ *    prefixed "[lgn] ": the kernel, tile size, grid and queue of a grouped call,
+ *    the selection path of a quantile, the closed forms' inputs and results, the
+ *    reason an argument was refused.  Device work is not affected.
  */
 #ifndef LGN_H
 #define LGN_H

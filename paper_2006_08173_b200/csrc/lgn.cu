@@ -9,6 +9,7 @@
 #include <cuda_runtime.h>
 
 #include "lgn.h"
+#include "lgn_log.h"
 #include "lgn_kernels.cuh"
 
 namespace lgn {
@@ -135,13 +136,20 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
     std::vector<uint64_t> ns(L);
     for (int k = 0; k < L; ++k) {
         lgn_status s = check_layer(layers[k].d);
-        if (s != LGN_OK) return s;
+        if (s != LGN_OK) {
+            log_line("layer %d of %d refused: %s (n=%llu dt=%d mode=%d nbits=%d S=%g)", k, L, lgn_status_string(s),
+                     (unsigned long long)layers[k].d.n, (int)layers[k].d.dt, (int)layers[k].d.mode, (int)layers[k].d.nbits, layers[k].d.S);
+            return s;
+        }
         ns[k] = layers[k].d.n;
     }
     WsLayout w;
     if (!ws_layout(ns.data(), L, w)) return LGN_ERR_UNSUPPORTED;
     if (ws == nullptr || !aligned16(ws)) return LGN_ERR_INVALID_ARG;
-    if (ws_bytes < w.total) return LGN_ERR_WORKSPACE;
+    if (ws_bytes < w.total) {
+        log_line("workspace of %zu bytes refused: %d layers need %zu", ws_bytes, L, (size_t)w.total);
+        return LGN_ERR_WORKSPACE;
+    }
 
     std::vector<LayerState> st(L);
     for (int k = 0; k < L; ++k) {
@@ -206,6 +214,18 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
         memset(&s, 0, sizeof s);
         s.first_item = total_items; s.ntiles = 0xFFFFFFFFu - total_items;
         segs.push_back(s);
+    }
+
+    if (log_enabled()) {
+        uint64_t elems = 0;
+        for (int k = 0; k < L; ++k) elems += st[k].n;
+        const int v = variant_of(st[0].mode, st[0].nbits, st[0].rounding);
+        log_line("grouped call: %d layers, %llu elements; kernel: %s%s (variant %d of %s), tiles of %u elements, grid %d x %d threads, "
+                 "%u queue items in %zu runs, counters %s, %d set-up launch(es), workspace %zu bytes",
+                 L, (unsigned long long)elems, fn == kCompressGeneral ? "general (layers differ)" : "specialised",
+                 (fn != kCompressGeneral && any_ext) ? " with extended statistics" : "", v, st[0].dt == LGN_BF16 ? "bf16" : "fp32",
+                 tile_elems, grid, kThreads, total_items, segs.size() - 1, st[0].counters ? "on" : "off",
+                 upload_launches(upload_bytes(w, L)), (size_t)w.total);
     }
 
     // image of [header | states | dyn (zero) | segments]
@@ -320,6 +340,8 @@ extern "C" lgn_status lgn_threshold(double mu, double sigma, double zero_frac, d
     if (!(S >= 0.0 && S < 1.0) || !(zero_frac >= 0.0 && zero_frac <= 1.0)) return LGN_ERR_INVALID_ARG;
     if (!std::isfinite(mu) || !(sigma >= 0.0) || !std::isfinite(sigma)) return LGN_ERR_INVALID_ARG;
     *tau = threshold_for(mu, sigma, zero_frac, S);
+    log_line("threshold: mu=%.17g sigma=%.17g zero fraction=%.17g S=%.17g -> S'=%.17g tau=%.17g", mu, sigma, zero_frac, S,
+             zero_frac < 1.0 ? (S - zero_frac) / (1.0 - zero_frac) : 0.0, *tau);
     return LGN_OK;
 }
 
@@ -335,6 +357,7 @@ extern "C" lgn_status lgn_fp_format(double mu, double sigma, int nbits, lgn_fp_f
     if (nbits < 4 || nbits > 8) return LGN_ERR_UNSUPPORTED;
     if (!std::isfinite(mu) || !(sigma >= 0.0) || !std::isfinite(sigma)) return LGN_ERR_INVALID_ARG;
     choose_format(mu, sigma, nbits, *fmt);
+    log_line("format: mu=%.17g sigma=%.17g nbits=%d -> 1-%d-%d, scale 2^%d", mu, sigma, nbits, fmt->exp_bits, fmt->man_bits, fmt->scale_exp);
     return LGN_OK;
 }
 

@@ -22,6 +22,7 @@
 #include "lgn.h"
 #include "lgn_closed_form.cuh"
 #include "lgn_device.cuh"
+#include "lgn_log.h"
 
 namespace lgn {
 
@@ -399,6 +400,9 @@ extern "C" lgn_status lgn_prefix_encode(const void *g, uint64_t n, lgn_dtype dt,
     unsigned long long *state = reinterpret_cast<unsigned long long *>(static_cast<char *>(ws) + sizeof(PfxCtl));
     #define LGN_PFX1(D, P) { const unsigned grid = resident_grid(prefix_encode_kernel<D, P>, nb); \
                              if (grid == 0) return LGN_ERR_CUDA; \
+                             log_line("prefix encoder: %llu blocks of %u elements, grid %u x %d threads, Eq. 5 %s, threshold from %s", \
+                                      (unsigned long long)nb, (unsigned)LGN_PREFIX_BLOCK, grid, kPfxThreads, P ? "applied" : "not applied", \
+                                      tau_from_dev ? "a result record on the device" : "the host"); \
                              prefix_encode_kernel<D, P><<<grid, kPfxThreads, 0, st>>>(g, n, nb, tau_used, tau_from_dev, seed, wy, \
                                  ctl, state, off_dev, stream_dev, capacity_words); }
     if (dt == LGN_F32) { if (apply_prune) LGN_PFX1(LGN_F32, true) else LGN_PFX1(LGN_F32, false) }

@@ -43,6 +43,7 @@
 
 #include "lgn.h"
 #include "lgn_device.cuh"
+#include "lgn_log.h"
 
 namespace lgn {
 
@@ -633,6 +634,10 @@ extern "C" lgn_status lgn_quantile(const void *g, uint64_t n, lgn_dtype dt, doub
         if (root * root > (double)elems) elems = (uint64_t)(root * root);
     }
     const int direct = n < kQDirect || elems > n / 8;
+    log_line("quantile: n=%llu %s q=%.17g -> %s", (unsigned long long)n, f32 ? "fp32" : "bf16", q,
+             direct ? (n < kQDirect ? "radix selection (tensor below 2^24 elements)" : "radix selection (the sample would pass n / 8)")
+                    : "one read around a bracket from a sample");
+    if (!direct) log_line("quantile: sample of %llu elements", (unsigned long long)elems);
     bool first = true, ok = true;                            // the first kernel of the call follows the memset in plain stream order
     auto launch = [&](const void *fn, unsigned blocks, unsigned threads, size_t shared, void **args) {
         cudaLaunchConfig_t cfg;

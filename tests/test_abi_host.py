@@ -254,3 +254,23 @@ def test_allocate_sparsity_agrees_with_oracle(lgn, oracle):
     with pytest.raises(lgn.LgnError):
         lgn.lgn_allocate_sparsity([dict(n=1, sigma=1.0, zero_frac=1.5)], 0, 0.5, 0.9)
     assert lgn.lgn_allocate_sparsity([], 0, 0.5, 0.9) == ([], 0.0)
+
+
+def test_lgn_log_prints_host_decisions():
+    """LGN_LOG=1: one "[lgn] " line per host-side decision on stderr; nothing without it."""
+    import os, subprocess, sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = ("from paper_2006_08173_b200 import binding as lgn\n"
+            "print(lgn.lgn_threshold(-12.0, 2.0, 0.4, 0.8))\n"
+            "print(lgn.lgn_fp_format(-12.0, 2.0, 6)['exp_bits'])\n")
+    def run(env_extra):
+        env = dict(os.environ); env.pop("LGN_LOG", None); env.update(env_extra)
+        return subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=300)
+    quiet = run({})
+    assert quiet.returncode == 0 and "[lgn]" not in quiet.stderr
+    assert "[lgn]" not in run({"LGN_LOG": "0"}).stderr
+    loud = run({"LGN_LOG": "1"})
+    assert loud.returncode == 0 and loud.stdout == quiet.stdout
+    lines = [l for l in loud.stderr.splitlines() if l.startswith("[lgn] ")]
+    assert any(l.startswith("[lgn] threshold: mu=-12 sigma=2 zero fraction=0.4") and "S'=0.66666" in l and "tau=" in l for l in lines)
+    assert any(l.startswith("[lgn] format: mu=-12 sigma=2 nbits=6 -> 1-") for l in lines)
