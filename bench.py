@@ -77,6 +77,9 @@ for _lg in (26, 28):
                                                          dtype="f32" if _dt == "fp32" else "bf16", mode="prefix")
         WORKLOADS[f"prefix_encode_{_dt}_2p{_lg}"] = dict(net="aux", kind="prefix", log2n=_lg,
                                                          dtype="f32" if _dt == "fp32" else "bf16", mode="prefix")
+for _dt in ("fp32", "bf16"):
+    WORKLOADS[f"quantile_{_dt}_2p30"] = dict(net="aux", kind="quantile", log2n=30,
+                                             dtype="f32" if _dt == "fp32" else "bf16", mode="quantile")
 
 
 def workload_specs(name: str, batch: int, seed: int):
