@@ -284,54 +284,74 @@ prefix_encode_kernel(const void *g, uint64_t n, uint64_t nblocks, float tau_host
 __global__ void prefix_empty_kernel(uint64_t *off) { off[0] = 0ull; }
 
 // One thread decodes one block (the code is sequential within a block); a warp takes 32
-// consecutive blocks.  Every lane decodes 32 elements of its block into a row of a
-// shared-memory tile, then the warp writes the 32 rows out, one coalesced store per row,
-// so that the output leaves in whole 128-byte (fp32) or 64-byte (bf16) pieces.  The next
-// stream word of a lane is loaded one refill ahead of its use.
+// consecutive blocks and moves in rounds of 32 elements per block.  Per round:
+//   1. the warp copies, row by row with coalesced loads, the next 40 words of each of its 32
+//      streams into shared memory (32 elements take at most 32 x 34 bits = 34 words, plus
+//      the two words a 64-bit window may reach past its first);
+//   2. every lane decodes 32 elements of its block from its row, without a branch: a 64-bit
+//      window at the current bit, the class from its two low bits, the value from the bits
+//      behind them, the length added to the bit position;
+//   3. the warp writes the 32 rows of decoded elements out, one coalesced store per row.
+// The re-read of words a slow stream has not consumed yet hits L1; no load sits on the
+// decode chain.
 constexpr int kDecThreads = 128;
+constexpr int kDecRowWords = 40;
 template <int DT>
 __global__ void __launch_bounds__(kDecThreads)
 prefix_decode_kernel(const uint32_t *stream, const uint64_t *off, uint64_t n, uint64_t nblocks, float tau_host,
                      const lgn_layer_result_t *tau_from, void *out) {
+    constexpr uint32_t W = PfxTraits<DT>::kWidth;
     __shared__ uint32_t tile[kDecThreads / 32][32][33];
+    __shared__ uint32_t rows[kDecThreads / 32][32][kDecRowWords + 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint64_t b0 = ((uint64_t)blockIdx.x * kDecThreads + threadIdx.x) & ~31ull;   // first block of this warp
     const uint64_t b = b0 + lane;
     if (b0 >= nblocks) return;                                   // whole warp
     const uint32_t tp = tau_pattern<DT>(pfx_tau(tau_host, tau_from));
     const bool live = b < nblocks;
-    const uint32_t *p = stream, *end = stream;
-    if (live) { p = stream + off[b]; end = stream + off[b + 1]; }
-    unsigned long long buf = 0ull;
-    int have = 0;
-    uint32_t ahead = p < end ? *p : 0u;                          // the word at p, already on its way
+    unsigned long long at = 0ull, end = 0ull;                    // this lane's stream: next word, one past its last word
+    if (live) { at = off[b]; end = off[b + 1]; }
+    uint32_t bit = 0u;                                           // bits of word `at` already consumed
     const uint64_t i0 = b * LGN_PREFIX_BLOCK;
     const uint64_t i1 = !live ? i0 : (i0 + LGN_PREFIX_BLOCK < n ? i0 + LGN_PREFIX_BLOCK : n);
-    auto refill = [&]() {                                        // keeps 33..64 bits in hand (zeros past the block)
-        if (have <= 32) {
-            buf |= (unsigned long long)ahead << have;
-            have += 32;
-            ++p;
-            ahead = p < end ? *p : 0u;
-        }
-    };
     for (uint32_t j = 0; j < LGN_PREFIX_BLOCK; j += 32) {
-        const uint64_t ic = i0 + j;
-        const uint32_t cnt = ic >= i1 ? 0u : (i1 - ic < 32u ? (uint32_t)(i1 - ic) : 32u);
-        for (uint32_t k = 0; k < cnt; ++k) {
-            refill();
-            uint32_t pat;
-            if ((buf & 1ull) == 0ull)      { pat = 0u; buf >>= 1; have -= 1; }
-            else if ((buf & 2ull) == 0ull) { pat = (buf & 4ull) ? (tp | PfxTraits<DT>::kSign) : tp; buf >>= 3; have -= 3; }
-            else {
-                buf >>= 2; have -= 2;
-                refill();                                        // now at least 32 bits: the whole value
-                pat = (uint32_t)buf & (DT == LGN_F32 ? 0xFFFFFFFFu : 0xFFFFu);
-                buf >>= PfxTraits<DT>::kWidth; have -= PfxTraits<DT>::kWidth;
+        // 1. rows: lane l fetches word l (and 32 + l) of every stream in turn
+        {
+            uint32_t first[32], more[32];                        // all 64 loads in flight together
+            #pragma unroll
+            for (int r = 0; r < 32; ++r) {
+                const unsigned long long ra = __shfl_sync(0xFFFFFFFFu, at, r), re = __shfl_sync(0xFFFFFFFFu, end, r);
+                first[r] = ra + lane < re ? __ldg(stream + ra + lane) : 0u;
+                more[r] = (lane < kDecRowWords - 32 && ra + 32u + lane < re) ? __ldg(stream + ra + 32u + lane) : 0u;
             }
-            tile[warp][lane][k] = pat;
+            #pragma unroll
+            for (int r = 0; r < 32; ++r) {
+                rows[warp][r][lane] = first[r];
+                if (lane < kDecRowWords - 32) rows[warp][r][32 + lane] = more[r];
+            }
         }
         __syncwarp();
+        // 2. decode
+        const uint64_t ic = i0 + j;
+        const uint32_t cnt = ic >= i1 ? 0u : (i1 - ic < 32u ? (uint32_t)(i1 - ic) : 32u);
+        const uint32_t *row = rows[warp][lane];
+        uint32_t pos = bit;
+        #pragma unroll 4
+        for (uint32_t k = 0; k < 32u; ++k) {
+            const uint32_t wi = pos >> 5, sh = pos & 31u;
+            const uint32_t a = row[wi], c = row[wi + 1], d = row[wi + 2];
+            const uint32_t lo = __funnelshift_r(a, c, sh), hi = __funnelshift_r(c, d, sh);     // 64 bits from the current bit
+            const uint32_t val = __funnelshift_r(lo, hi, 2) & (DT == LGN_F32 ? 0xFFFFFFFFu : 0xFFFFu);
+            const bool nz = (lo & 1u) != 0u, isval = (lo & 2u) != 0u;
+            const uint32_t alpha = (lo & 4u) ? (tp | PfxTraits<DT>::kSign) : tp;
+            const uint32_t pat = nz ? (isval ? val : alpha) : 0u;
+            const uint32_t len = nz ? (isval ? 2u + W : 3u) : 1u;
+            if (k < cnt) { tile[warp][lane][k] = pat; pos += len; }
+        }
+        at += pos >> 5;
+        bit = pos & 31u;
+        __syncwarp();
+        // 3. rows of elements out
         #pragma unroll 4
         for (int r = 0; r < 32; ++r) {                           // row r = block b0 + r, elements j .. j+31
             const uint64_t i = (b0 + r) * LGN_PREFIX_BLOCK + j + lane;
