@@ -309,8 +309,12 @@ prefix_decode_kernel(const uint32_t *stream, const uint64_t *off, uint64_t n, ui
     if (b0 >= nblocks) return;                                   // whole warp
     const uint32_t tp = tau_pattern<DT>(pfx_tau(tau_host, tau_from));
     const bool live = b < nblocks;
-    unsigned long long at = 0ull, end = 0ull;                    // this lane's stream: next word, one past its last word
-    if (live) { at = off[b]; end = off[b + 1]; }
+    // this lane's stream: next word and one past its last word, counted from the warp's first word
+    // (32 blocks are at most 32 x 2176 words long: 32 bits do)
+    const unsigned long long w0 = off[b0];
+    const uint32_t *base = stream + w0;
+    uint32_t at = 0u, end = 0u;
+    if (live) { at = (uint32_t)(off[b] - w0); end = (uint32_t)(off[b + 1] - w0); }
     uint32_t bit = 0u;                                           // bits of word `at` already consumed
     const uint64_t i0 = b * LGN_PREFIX_BLOCK;
     const uint64_t i1 = !live ? i0 : (i0 + LGN_PREFIX_BLOCK < n ? i0 + LGN_PREFIX_BLOCK : n);
@@ -320,9 +324,9 @@ prefix_decode_kernel(const uint32_t *stream, const uint64_t *off, uint64_t n, ui
             uint32_t first[32], more[32];                        // all 64 loads in flight together
             #pragma unroll
             for (int r = 0; r < 32; ++r) {
-                const unsigned long long ra = __shfl_sync(0xFFFFFFFFu, at, r), re = __shfl_sync(0xFFFFFFFFu, end, r);
-                first[r] = ra + lane < re ? __ldg(stream + ra + lane) : 0u;
-                more[r] = (lane < kDecRowWords - 32 && ra + 32u + lane < re) ? __ldg(stream + ra + 32u + lane) : 0u;
+                const uint32_t ra = __shfl_sync(0xFFFFFFFFu, at, r) + lane, re = __shfl_sync(0xFFFFFFFFu, end, r);
+                first[r] = ra < re ? __ldg(base + ra) : 0u;
+                more[r] = (lane < kDecRowWords - 32 && ra + 32u < re) ? __ldg(base + ra + 32u) : 0u;
             }
             #pragma unroll
             for (int r = 0; r < 32; ++r) {
@@ -339,7 +343,7 @@ prefix_decode_kernel(const uint32_t *stream, const uint64_t *off, uint64_t n, ui
         #pragma unroll 4
         for (uint32_t k = 0; k < 32u; ++k) {
             const uint32_t wi = pos >> 5, sh = pos & 31u;
-            const uint32_t a = row[wi], c = row[wi + 1], d = row[wi + 2];
+            const uint32_t a = row[wi], c = row[wi + 1], d = DT == LGN_F32 ? row[wi + 2] : 0u;  // bf16: 18 bits from bit 31 at most
             const uint32_t lo = __funnelshift_r(a, c, sh), hi = __funnelshift_r(c, d, sh);     // 64 bits from the current bit
             const uint32_t val = __funnelshift_r(lo, hi, 2) & (DT == LGN_F32 ? 0xFFFFFFFFu : 0xFFFFu);
             const bool nz = (lo & 1u) != 0u, isval = (lo & 2u) != 0u;
