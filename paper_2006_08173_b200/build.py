@@ -15,7 +15,7 @@ _CSRC = os.path.join(_PKG, "csrc")
 _OBJ = os.path.join(_PKG, "_build")
 LIB_PATH = os.path.join(_PKG, "liblgn.so")
 SOURCES = [os.path.join(_CSRC, f) for f in (
-    "lgn.cu", "lgn_inst_f32.cu", "lgn_inst_bf16.cu", "lgn_inst_bf16_big.cu", "lgn_inst_misc.cu",
+    "lgn.cu", "lgn_inst_f32.cu", "lgn_inst_bf16.cu", "lgn_inst_bf16_big.cu", "lgn_inst_f32_small.cu", "lgn_inst_bf16_small.cu", "lgn_inst_misc.cu",
     "lgn_prefix.cu", "lgn_dequant.cu", "lgn_quantile.cu", "lgn_host.cu")]
 _HEADERS = [os.path.join(_CSRC, "lgn_kernels.cuh"), os.path.join(_CSRC, "lgn_device.cuh"),
             os.path.join(_CSRC, "lgn_closed_form.cuh"), os.path.join(_ROOT, "include", "lgn.h")]

@@ -199,6 +199,19 @@ static lgn_status run_layers(const std::vector<InternalLayer> &layers, void *ws,
             if (grid < 1) return LGN_ERR_CUDA;
         }
     }
+    // Small calls (fewer standard tiles than CTAs; see kSmallCallTiles): smaller tiles.
+    if (fn != kCompressGeneral && tile_elems == kTileElems && !withhold_tile) {
+        uint64_t std_tiles = 0;
+        for (int k = 0; k < L; ++k) std_tiles += (st[k].n + kTileElems - 1) / kTileElems;
+        if (std_tiles < kSmallCallTiles && std_tiles < (uint64_t)grid) {
+            const void *const *from = compress_table(st[0].dt);
+            const void *const *to = st[0].dt == LGN_BF16 ? kCompressTableBf16Small : kCompressTableF32Small;
+            for (int v = 0; v < kVariants; ++v)
+                if (from[v] == fn) { fn = to[v]; tile_elems = st[0].dt == LGN_BF16 ? kSmallTileElemsBf16 : kSmallTileElemsF32; break; }
+            grid = persistent_ctas(fn);
+            if (grid < 1) return LGN_ERR_CUDA;
+        }
+    }
     uint32_t partial0 = 0;
     for (int k = 0; k < L; ++k) {
         LayerState &s = st[k];

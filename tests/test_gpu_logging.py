@@ -1,6 +1,7 @@
 """LGN_LOG=1 on a GPU machine: the host side reports which kernel, tile size, grid and queue a grouped
 call takes, and which selection path a quantile takes; the results are the same with and without it."""
 import os
+import re
 import subprocess
 import sys
 
@@ -46,8 +47,11 @@ def test_log_lines_of_a_grouped_call_and_a_quantile():
     lines = [l for l in loud.stderr.splitlines() if l.startswith("[lgn] ")]
     grouped = [l for l in lines if l.startswith("[lgn] grouped call: 2 layers, 370001 elements; kernel: specialised")]
     assert len(grouped) == 1
-    assert "of fp32" in grouped[0] and "tiles of 32768 elements" in grouped[0] and "x 256 threads" in grouped[0]
-    assert "26 queue items in" in grouped[0] and "counters off" in grouped[0]       # 10 + 3 tiles of statistics and as many of apply
+    assert "of fp32" in grouped[0] and "x 256 threads" in grouped[0] and "counters off" in grouped[0]
+    tile = int(re.search(r"tiles of (\d+) elements", grouped[0]).group(1))
+    assert tile in (8192, 32768)                                     # a call this small takes the small tiles
+    items = 2 * (-(-300_001 // tile) + -(-70_000 // tile))           # every tile once for statistics, once for apply
+    assert f"{items} queue items in" in grouped[0]
     assert any("quantile: n=300001 fp32" in l and "radix selection (tensor below 2^24 elements)" in l for l in lines)
     assert any("quantile: n=16777219 bf16" in l and "one read around a bracket from a sample" in l for l in lines)
     assert any("quantile: sample of 2097152 elements" in l for l in lines)
