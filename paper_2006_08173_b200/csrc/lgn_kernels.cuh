@@ -103,22 +103,26 @@ struct WsLayout {
 static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Tiles of small calls.  A call of fewer tiles than the grid has CTAs cannot fill the GPU: each of its
-// CTAs streams one 128 KiB tile alone, bound by the latency of its own loads.  Such calls take tiles of a
-// quarter of the bytes (a flat 2^20-element fp32 tensor: 128 CTAs of 32 KiB instead of 32 of 128 KiB).
+// CTAs streams one 128 KiB tile alone, bound by the latency of its own loads; a call of little more than
+// one round of the grid ends each pass with a second round that few CTAs run.  Such calls (fewer tiles than
+// one and a half rounds) take tiles of a quarter of the bytes (a flat 2^20-element fp32 tensor: 128 CTAs of
+// 32 KiB instead of 32 of 128 KiB).
 // kSmallCallTiles bounds "small" for the workspace layout, which knows no device: below it the layout has
 // room for the small tiles' partial sums, and the kernels are chosen by the actual grid, never above it.
 constexpr int kSmallTileElemsF32 = kTileElems / 4, kSmallTileElemsBf16 = kTileElems / 2;
-constexpr uint64_t kSmallCallTiles = 512;
+constexpr uint64_t kSmallCallTiles = 1024;
 
 static bool ws_layout(const uint64_t *n_per_layer, int L, WsLayout &w) {
     if (L < 0) return false;
-    uint64_t tiles = 0, small_tiles = 0;
+    uint64_t tiles = 0;
     for (int k = 0; k < L; ++k) {
         if (n_per_layer[k] > (1ull << 44)) return false;
         tiles += (n_per_layer[k] + kTileElems - 1) / kTileElems;
-        small_tiles += (n_per_layer[k] + kSmallTileElemsF32 - 1) / kSmallTileElemsF32;
     }
-    if (tiles < kSmallCallTiles) tiles = small_tiles;
+    // Room for the partial sums of small tiles: a small call has at most four times its standard tiles,
+    // so three times kSmallCallTiles more slots serve every small call; added to every layout, so that the
+    // workspace of a list of layers is enough for any subset of it (the host-buffer form runs subsets).
+    tiles += 3 * kSmallCallTiles;
     if (tiles >= (1ull << 31)) return false;
     w.total_tiles = tiles;
     w.nseg_max = 2u * (uint32_t)L + 2u;
